@@ -1,0 +1,444 @@
+// C ABI of the Flora hot path (see include/flora.h for the contract of every entry point).
+// This file validates arguments, picks a kernel family and launches; all arithmetic of the path
+// lives in the kernels of flora_simt.cuh (fp32 SIMT) and flora_tc.cuh (tcgen05 tensor cores).
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <atomic>
+#include <new>
+#include <vector>
+
+#include "../../include/flora.h"
+#include "flora_rng.cuh"
+#include "flora_simt.cuh"
+#include "flora_tc.cuh"
+
+using namespace flora;
+
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+std::atomic<int> g_force_path{0};
+
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+inline flora_status launched()
+{
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaPeekAtLastError() == cudaSuccess ? FLORA_OK : FLORA_ERR_CUDA;
+}
+inline float projection_scale(int r) { return 1.0f / sqrtf((float)r); }
+inline size_t elem_size(int32_t dt) { return dt == FLORA_BF16 ? 2 : 4; }
+
+flora_status check_mat(const flora_mat* a, bool f32_only)
+{
+    if (!a) return FLORA_ERR_NULL;
+    if (a->dtype != FLORA_F32 && a->dtype != FLORA_BF16) return FLORA_ERR_DTYPE;
+    if (f32_only && a->dtype != FLORA_F32) return FLORA_ERR_DTYPE;
+    if (a->rows < 0 || a->cols < 0 || a->ld < a->cols) return FLORA_ERR_SHAPE;
+    if (a->rows > 0 && a->cols > 0) {
+        if (!a->data) return FLORA_ERR_NULL;
+        if (reinterpret_cast<uintptr_t>(a->data) % elem_size(a->dtype)) return FLORA_ERR_ALIGN;
+    }
+    return FLORA_OK;
+}
+
+// G (or W) against its sketch: same row count, rank in range.
+flora_status check_pair(const flora_mat* big, const flora_mat* sketch)
+{
+    flora_status st = check_mat(big, false);
+    if (st) return st;
+    st = check_mat(sketch, true);
+    if (st) return st;
+    if (sketch->cols < 1 || sketch->cols > 256) return FLORA_ERR_RANK;
+    if (sketch->rows != big->rows) return FLORA_ERR_SHAPE;
+    if (big->cols > (int64_t)4 * 0x7FFFFFFF || big->rows > 0x7FFFFFFFll * 32) return FLORA_ERR_UNSUPPORTED;
+    return FLORA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// SIMT launches
+// ------------------------------------------------------------------------------------------------
+flora_status simt_compress(const flora_mat* G, flora_mat* S, uint64_t seed, float a, float b, cudaStream_t st)
+{
+    const int r = (int)S->cols;
+    if (G->rows == 0) return FLORA_OK;
+    const unsigned grid = (unsigned)((G->rows + 31) / 32);
+    if (G->dtype == FLORA_BF16)
+        simt_compress_kernel<__nv_bfloat16><<<grid, SIMT_THREADS, 0, st>>>(
+            (const __nv_bfloat16*)G->data, G->rows, G->cols, G->ld, (float*)S->data, S->ld, r, make_key(seed),
+            projection_scale(r), a, b);
+    else
+        simt_compress_kernel<float><<<grid, SIMT_THREADS, 0, st>>>(
+            (const float*)G->data, G->rows, G->cols, G->ld, (float*)S->data, S->ld, r, make_key(seed),
+            projection_scale(r), a, b);
+    return launched();
+}
+
+flora_status simt_decompress(flora_mat* W, const flora_mat* C, uint64_t seed, float step, cudaStream_t st)
+{
+    const int r = (int)C->cols;
+    if (W->rows == 0 || W->cols == 0) return FLORA_OK;
+    dim3 grid((unsigned)((W->cols + 63) / 64), (unsigned)((W->rows + 31) / 32));
+    if (grid.y > 65535) return FLORA_ERR_UNSUPPORTED;
+    if (W->dtype == FLORA_BF16)
+        simt_decompress_kernel<__nv_bfloat16><<<grid, SIMT_THREADS, 0, st>>>(
+            (__nv_bfloat16*)W->data, W->rows, W->cols, W->ld, (const float*)C->data, C->ld, r, make_key(seed),
+            projection_scale(r), step);
+    else
+        simt_decompress_kernel<float><<<grid, SIMT_THREADS, 0, st>>>(
+            (float*)W->data, W->rows, W->cols, W->ld, (const float*)C->data, C->ld, r, make_key(seed),
+            projection_scale(r), step);
+    return launched();
+}
+
+// T (r x r, zeroed here) <- A_old A_new^T with the SIMT kernel.
+flora_status simt_gram(float* T, int r, int64_t m, int32_t operand, uint64_t s_old, uint64_t s_new, cudaStream_t st)
+{
+    if (cudaMemsetAsync(T, 0, sizeof(float) * r * r, st) != cudaSuccess) return FLORA_ERR_CUDA;
+    if (m == 0) return FLORA_OK;
+    const int tiles = (r + 31) / 32;
+    int64_t splits = (m + 511) / 512;
+    if (splits > 1024) splits = 1024;
+    int64_t kper = ((m + splits - 1) / splits + 31) / 32 * 32;
+    splits = (m + kper - 1) / kper;
+    dim3 grid((unsigned)(tiles * tiles), (unsigned)splits);
+    simt_gram_kernel<<<grid, SIMT_THREADS, 0, st>>>(T, r, m, kper, operand == FLORA_BF16, make_key(s_old),
+                                                    make_key(s_new), projection_scale(r));
+    return launched();
+}
+
+flora_status simt_apply_gram(flora_mat* dst, const flora_mat* src, const float* T, float a, float b, cudaStream_t st)
+{
+    if (dst->rows == 0) return FLORA_OK;
+    const unsigned grid = (unsigned)((dst->rows + 7) / 8);
+    simt_apply_gram_kernel<<<grid, SIMT_THREADS, 0, st>>>((float*)dst->data, dst->ld, (const float*)src->data, src->ld,
+                                                          dst->rows, (int)dst->cols, T, a, b);
+    return launched();
+}
+
+flora_status check_transfer(const flora_mat* dst, const flora_mat* src, int64_t m, int32_t operand)
+{
+    flora_status st = check_mat(dst, true);
+    if (st) return st;
+    st = check_mat(src, true);
+    if (st) return st;
+    if (operand != FLORA_F32 && operand != FLORA_BF16) return FLORA_ERR_DTYPE;
+    if (dst->cols < 1 || dst->cols > 256 || src->cols != dst->cols) return FLORA_ERR_RANK;
+    if (src->rows != dst->rows || m < 0 || m > (int64_t)4 * 0x7FFFFFFF) return FLORA_ERR_SHAPE;
+    return FLORA_OK;
+}
+
+// dst <- b dst + a src (A_old A_new^T) with T in the given scratch (r*r floats).
+flora_status transfer_with_scratch(flora_mat* dst, const flora_mat* src, int64_t m, int32_t operand, uint64_t s_old,
+                                   uint64_t s_new, float a, float b, float* T, cudaStream_t st)
+{
+    flora_status rc = simt_gram(T, (int)dst->cols, m, operand, s_old, s_new, st);
+    if (rc) return rc;
+    return simt_apply_gram(dst, src, T, a, b, st);
+}
+
+bool use_tc(const flora_mat* big, const flora_mat* sketch)
+{
+    if (g_force_path.load(std::memory_order_relaxed) == 1) return false;
+    return tc_supported(big, sketch);
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+// set object
+// ------------------------------------------------------------------------------------------------
+struct flora_set {
+    std::vector<flora_mat> G, W, S;
+    int r = 0;
+    bool has_G = false, has_W = false;
+    TcSet tc;   // tensor-core work lists and descriptors (empty when the set is not eligible)
+};
+
+extern "C" {
+
+flora_status flora_compress_accumulate(const flora_mat* G, flora_mat* C, uint64_t seed, int r, void* stream)
+{
+    flora_status st = check_pair(G, C);
+    if (st) return st;
+    if (r != C->cols) return FLORA_ERR_RANK;
+    if (G->rows == 0 || G->cols == 0) return FLORA_OK;
+    if (use_tc(G, C)) return tc_compress_single(G, C, seed, 1.0f, 1.0f, as_stream(stream), g_launches);
+    return simt_compress(G, C, seed, 1.0f, 1.0f, as_stream(stream));
+}
+
+flora_status flora_momentum_step(const flora_mat* G, flora_mat* M, float beta, uint64_t seed, void* stream)
+{
+    flora_status st = check_pair(G, M);
+    if (st) return st;
+    if (G->rows == 0) return FLORA_OK;
+    if (G->cols > 0 && use_tc(G, M)) return tc_compress_single(G, M, seed, 1.0f - beta, beta, as_stream(stream), g_launches);
+    return simt_compress(G, M, seed, 1.0f - beta, beta, as_stream(stream));
+}
+
+flora_status flora_decompress_apply(flora_mat* W, const flora_mat* C, uint64_t seed, float lr, float scale, void* stream)
+{
+    flora_status st = check_pair(W, C);
+    if (st) return st;
+    if (W->rows == 0 || W->cols == 0) return FLORA_OK;
+    if (use_tc(W, C)) return tc_decompress_single(W, C, seed, lr * scale, as_stream(stream), g_launches);
+    return simt_decompress(W, C, seed, lr * scale, as_stream(stream));
+}
+
+flora_status flora_transfer_axpby(flora_mat* dst, const flora_mat* src, int64_t m, int32_t operand, uint64_t seed_old,
+                                  uint64_t seed_new, float a, float b, void* stream)
+{
+    flora_status st = check_transfer(dst, src, m, operand);
+    if (st) return st;
+    if (dst->rows == 0) return FLORA_OK;
+    const int r = (int)dst->cols;
+    float* T = nullptr;
+    if (cudaMallocAsync((void**)&T, sizeof(float) * r * r, as_stream(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return FLORA_ERR_ALLOC;
+    }
+    st = transfer_with_scratch(dst, src, m, operand, seed_old, seed_new, a, b, T, as_stream(stream));
+    if (cudaFreeAsync(T, as_stream(stream)) != cudaSuccess && st == FLORA_OK) st = FLORA_ERR_CUDA;
+    return st;
+}
+
+flora_status flora_resample_transfer(flora_mat* M, int64_t m, int32_t operand, uint64_t seed_old, uint64_t seed_new, void* stream)
+{
+    return flora_transfer_axpby(M, M, m, operand, seed_old, seed_new, 1.0f, 0.0f, stream);
+}
+
+flora_status flora_materialize_A(flora_mat* out, uint64_t seed, void* stream)
+{
+    flora_status st = check_mat(out, false);
+    if (st) return st;
+    if (out->rows < 1 || out->rows > 256) return FLORA_ERR_RANK;
+    if (out->cols == 0) return FLORA_OK;
+    if (out->cols > (int64_t)4 * 0x7FFFFFFF) return FLORA_ERR_UNSUPPORTED;
+    const int r = (int)out->rows;
+    const int64_t tasks = (out->cols + 3) / 4 * r;
+    const unsigned grid = (unsigned)((tasks + 255) / 256);
+    if (out->dtype == FLORA_BF16)
+        materialize_kernel<__nv_bfloat16><<<grid, 256, 0, as_stream(stream)>>>((__nv_bfloat16*)out->data, r, out->cols, out->ld,
+                                                                              make_key(seed), projection_scale(r));
+    else
+        materialize_kernel<float><<<grid, 256, 0, as_stream(stream)>>>((float*)out->data, r, out->cols, out->ld, make_key(seed),
+                                                                      projection_scale(r));
+    return launched();
+}
+
+// ------------------------------------------------------------------------------------------------
+// sets
+// ------------------------------------------------------------------------------------------------
+flora_status flora_set_create(int count, const flora_mat* G, const flora_mat* W, const flora_mat* S, flora_set** out)
+{
+    if (!out || !S || (!G && !W)) return FLORA_ERR_NULL;
+    if (count < 0) return FLORA_ERR_SHAPE;
+    *out = nullptr;
+    int r = count ? (int)S[0].cols : 1;
+    for (int i = 0; i < count; ++i) {
+        const flora_mat* big = G ? &G[i] : &W[i];
+        flora_status st = check_pair(big, &S[i]);
+        if (st) return st;
+        if (S[i].cols != r) return FLORA_ERR_RANK;
+        if (G && W) {
+            st = check_pair(&W[i], &S[i]);
+            if (st) return st;
+            if (W[i].cols != G[i].cols) return FLORA_ERR_SHAPE;
+            if (W[i].dtype != G[i].dtype) return FLORA_ERR_DTYPE;
+        }
+    }
+    flora_set* s = new (std::nothrow) flora_set();
+    if (!s) return FLORA_ERR_ALLOC;
+    s->r = r;
+    s->has_G = G != nullptr;
+    s->has_W = W != nullptr;
+    s->S.assign(S, S + count);
+    if (G) s->G.assign(G, G + count);
+    if (W) s->W.assign(W, W + count);
+    flora_status st = tc_set_build(s->tc, s->G, s->W, s->S);
+    if (st) {
+        tc_set_free(s->tc);
+        delete s;
+        return st;
+    }
+    *out = s;
+    return FLORA_OK;
+}
+
+flora_status flora_set_destroy(flora_set* set)
+{
+    if (!set) return FLORA_OK;
+    tc_set_free(set->tc);
+    delete set;
+    return FLORA_OK;
+}
+
+flora_status flora_set_rebind_gradients(flora_set* set, const flora_mat* G)
+{
+    if (!set || !G) return FLORA_ERR_NULL;
+    if (!set->has_G) return FLORA_ERR_UNSUPPORTED;
+    for (size_t i = 0; i < set->G.size(); ++i) {
+        flora_status st = check_mat(&G[i], false);
+        if (st) return st;
+        if (G[i].rows != set->G[i].rows || G[i].cols != set->G[i].cols || G[i].ld != set->G[i].ld) return FLORA_ERR_SHAPE;
+        if (G[i].dtype != set->G[i].dtype) return FLORA_ERR_DTYPE;
+    }
+    std::vector<flora_mat> newG(G, G + set->G.size());
+    flora_status st = tc_set_rebind(set->tc, newG, set->S);
+    if (st) return st;
+    set->G.swap(newG);
+    return FLORA_OK;
+}
+
+static flora_status set_compress(flora_set* set, const uint64_t* seeds, float a, float b, void* stream)
+{
+    if (!set || !seeds) return FLORA_ERR_NULL;
+    if (!set->has_G) return FLORA_ERR_UNSUPPORTED;
+    if (set->tc.compress_ready && g_force_path.load() != 1)
+        return tc_set_compress(set->tc, seeds, a, b, as_stream(stream), g_launches);
+    for (size_t i = 0; i < set->G.size(); ++i) {
+        if (set->G[i].rows == 0) continue;
+        flora_status st = simt_compress(&set->G[i], &set->S[i], seeds[i], a, b, as_stream(stream));
+        if (st) return st;
+    }
+    return FLORA_OK;
+}
+
+flora_status flora_set_compress_accumulate(flora_set* set, const uint64_t* seeds, void* stream)
+{
+    return set_compress(set, seeds, 1.0f, 1.0f, stream);
+}
+
+flora_status flora_set_momentum_step(flora_set* set, float beta, const uint64_t* seeds, void* stream)
+{
+    return set_compress(set, seeds, 1.0f - beta, beta, stream);
+}
+
+flora_status flora_set_decompress_apply(flora_set* set, const uint64_t* seeds, float lr, float scale, void* stream)
+{
+    if (!set || !seeds) return FLORA_ERR_NULL;
+    if (!set->has_W) return FLORA_ERR_UNSUPPORTED;
+    if (set->tc.decompress_ready && g_force_path.load() != 1)
+        return tc_set_decompress(set->tc, seeds, lr * scale, as_stream(stream), g_launches);
+    for (size_t i = 0; i < set->W.size(); ++i) {
+        if (set->W[i].rows == 0 || set->W[i].cols == 0) continue;
+        flora_status st = simt_decompress(&set->W[i], &set->S[i], seeds[i], lr * scale, as_stream(stream));
+        if (st) return st;
+    }
+    return FLORA_OK;
+}
+
+flora_status flora_set_resample_transfer(flora_set* set, const uint64_t* seeds_old, const uint64_t* seeds_new, void* stream)
+{
+    if (!set || !seeds_old || !seeds_new) return FLORA_ERR_NULL;
+    const std::vector<flora_mat>& big = set->has_G ? set->G : set->W;
+    const int r = set->r;
+    float* T = nullptr;
+    if (set->S.empty()) return FLORA_OK;
+    if (cudaMallocAsync((void**)&T, sizeof(float) * r * r, as_stream(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return FLORA_ERR_ALLOC;
+    }
+    flora_status st = FLORA_OK;
+    for (size_t i = 0; i < set->S.size() && st == FLORA_OK; ++i) {
+        if (set->S[i].rows == 0) continue;
+        st = transfer_with_scratch(&set->S[i], &set->S[i], big[i].cols, big[i].dtype, seeds_old[i], seeds_new[i], 1.0f,
+                                   0.0f, T, as_stream(stream));
+    }
+    if (cudaFreeAsync(T, as_stream(stream)) != cudaSuccess && st == FLORA_OK) st = FLORA_ERR_CUDA;
+    return st;
+}
+
+flora_status flora_set_zero_state(flora_set* set, void* stream)
+{
+    if (!set) return FLORA_ERR_NULL;
+    for (auto& s : set->S) {
+        if (s.rows == 0) continue;
+        cudaError_t e = cudaMemset2DAsync(s.data, sizeof(float) * s.ld, 0, sizeof(float) * s.cols, (size_t)s.rows, as_stream(stream));
+        if (e != cudaSuccess) return FLORA_ERR_CUDA;
+    }
+    return FLORA_OK;
+}
+
+flora_status flora_set_compress_accumulate_from_host(flora_set* set, const void* const* host_G, const uint64_t* seeds, void* stream)
+{
+    if (!set || !host_G || !seeds) return FLORA_ERR_NULL;
+    if (!set->has_G) return FLORA_ERR_UNSUPPORTED;
+    for (size_t i = 0; i < set->G.size(); ++i) {
+        const flora_mat& g = set->G[i];
+        if (g.rows == 0 || g.cols == 0) continue;
+        if (!host_G[i]) return FLORA_ERR_NULL;
+        const size_t es = elem_size(g.dtype);
+        cudaError_t e = cudaMemcpy2DAsync(g.data, es * g.ld, host_G[i], es * g.cols, es * g.cols, (size_t)g.rows,
+                                          cudaMemcpyHostToDevice, as_stream(stream));
+        if (e != cudaSuccess) return FLORA_ERR_CUDA;
+    }
+    return flora_set_compress_accumulate(set, seeds, stream);
+}
+
+flora_status flora_set_read_weights_to_host(flora_set* set, void* const* host_W, void* stream)
+{
+    if (!set || !host_W) return FLORA_ERR_NULL;
+    if (!set->has_W) return FLORA_ERR_UNSUPPORTED;
+    for (size_t i = 0; i < set->W.size(); ++i) {
+        const flora_mat& w = set->W[i];
+        if (w.rows == 0 || w.cols == 0) continue;
+        if (!host_W[i]) return FLORA_ERR_NULL;
+        const size_t es = elem_size(w.dtype);
+        cudaError_t e = cudaMemcpy2DAsync(host_W[i], es * w.cols, w.data, es * w.ld, es * w.cols, (size_t)w.rows,
+                                          cudaMemcpyDeviceToHost, as_stream(stream));
+        if (e != cudaSuccess) return FLORA_ERR_CUDA;
+    }
+    return FLORA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// host sequencing
+// ------------------------------------------------------------------------------------------------
+uint64_t flora_derive_seed(uint64_t base, uint64_t matrix, uint64_t epoch)
+{
+    uint64_t z = base ^ (matrix * 0x9E3779B97F4A7C15ull) ^ (epoch * 0xD1B54A32D192ED03ull);
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+int flora_resamples_at(int64_t t, int64_t kappa) { return (kappa > 0 && t >= 0 && t % kappa == 0) ? 1 : 0; }
+
+// ------------------------------------------------------------------------------------------------
+// diagnostics
+// ------------------------------------------------------------------------------------------------
+void flora_debug_force_path(int path) { g_force_path.store(path == 1 ? 1 : 0); }
+uint64_t flora_launch_count(void) { return g_launches.load(); }
+
+flora_status flora_device_status(void)
+{
+    int word = 0;
+    if (!tc_read_and_clear_error(&word)) return FLORA_ERR_CUDA;
+    return word ? FLORA_ERR_TIMEOUT : FLORA_OK;
+}
+
+const char* flora_status_string(flora_status s)
+{
+    switch (s) {
+        case FLORA_OK: return "ok";
+        case FLORA_ERR_NULL: return "null pointer";
+        case FLORA_ERR_SHAPE: return "bad shape or leading dimension";
+        case FLORA_ERR_DTYPE: return "dtype not allowed here";
+        case FLORA_ERR_ALIGN: return "misaligned pointer";
+        case FLORA_ERR_RANK: return "rank out of range or inconsistent";
+        case FLORA_ERR_CUDA: return "CUDA call failed";
+        case FLORA_ERR_TIMEOUT: return "device-side wait timed out";
+        case FLORA_ERR_UNSUPPORTED: return "unsupported arguments";
+        case FLORA_ERR_ALLOC: return "allocation failed";
+    }
+    return "unknown status";
+}
+
+int flora_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,68 @@
+"""Host sequencing of Algorithms 1 and 2: which call happens when, with which seed.
+
+Nothing here computes on matrices; the classes drive an object with the methods of
+:class:`paper_2402_03293_b200.binding.FloraSet` and ask the library for seeds
+(``flora_derive_seed``) and for the resampling schedule (``flora_resamples_at``).
+"""
+from __future__ import annotations
+
+from typing import List
+
+from . import binding
+
+
+class AccumulationCycle:
+    """Algorithm 1: tau compressions into C with one projection per matrix, then one decompression
+    with scale 1/tau; after that C is zeroed and the projection resampled (Section 2.4)."""
+
+    def __init__(self, ops, count: int, tau: int, base_seed: int = 0):
+        if tau < 1:
+            raise ValueError("tau must be positive")
+        self.ops, self.count, self.tau, self.base_seed = ops, count, tau, base_seed
+        self.epoch = 0
+        self.micro_step = 0
+
+    def seeds(self) -> List[int]:
+        return [binding.flora_derive_seed(self.base_seed, i, self.epoch) for i in range(self.count)]
+
+    def accumulate(self, stream=None) -> bool:
+        """Compress the gradients currently bound to the set; True when the cycle is full."""
+        if self.micro_step >= self.tau:
+            raise RuntimeError("cycle is full: call apply() first")
+        self.ops.compress_accumulate(self.seeds(), stream)
+        self.micro_step += 1
+        return self.micro_step == self.tau
+
+    def apply(self, lr: float, stream=None) -> None:
+        """Decompress the mean of the cycle into the weights, then start the next cycle."""
+        if self.micro_step != self.tau:
+            raise RuntimeError("cycle is not full")
+        self.ops.decompress_apply(self.seeds(), lr, 1.0 / self.tau, stream)
+        self.ops.zero_state(stream)
+        self.epoch += 1
+        self.micro_step = 0
+
+
+class MomentumState:
+    """Algorithm 2: at steps t = 0 mod kappa the projection is resampled and M is carried over by
+    M <- M A_old A_new^T; then M <- beta M + (1-beta) G A_new^T and the update M A_new is applied."""
+
+    def __init__(self, ops, count: int, beta: float, kappa: int, base_seed: int = 0, skip_transfer_of_zero_state: bool = True):
+        self.ops, self.count, self.beta, self.kappa, self.base_seed = ops, count, beta, kappa, base_seed
+        self.t = 0
+        self.epoch = 0
+        self.skip0 = skip_transfer_of_zero_state
+
+    def seeds(self, epoch: int) -> List[int]:
+        return [binding.flora_derive_seed(self.base_seed, i, epoch) for i in range(self.count)]
+
+    def step(self, lr: float, stream=None) -> None:
+        if binding.flora_resamples_at(self.t, self.kappa):
+            old, new = self.seeds(self.epoch), self.seeds(self.epoch + 1)
+            if not (self.t == 0 and self.skip0):          # M = 0 at t = 0: the transfer of zeros is zeros
+                self.ops.resample_transfer(old, new, stream)
+            self.epoch += 1
+        cur = self.seeds(self.epoch)
+        self.ops.momentum_step(self.beta, cur, stream)
+        self.ops.decompress_apply(cur, lr, 1.0, stream)
+        self.t += 1

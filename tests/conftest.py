@@ -8,3 +8,8 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200) and the built CUDA library")
+    # the C-ABI library and the oracle are built in-tree when missing or stale (nvcc / gcc, no GPU needed)
+    from paper_2402_03293_b200 import _build
+    from oracle import flora_oracle
+    _build.build()
+    flora_oracle.build()

@@ -1,0 +1,243 @@
+"""GPU parity: every operation of the C ABI against the CPU oracle on the same stored inputs.
+
+Bit-exact for the generated projection; max |x-ref| / max |ref| <= 1e-5 (fp32) or 2e-2 (bf16
+inputs, fp32 accumulation) for the contractions."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import flora_oracle as orc
+from paper_2402_03293_b200 import binding as fb
+from paper_2402_03293_b200 import workloads as wl
+from tests.parity_util import (TOL, oracle_compress, oracle_decompress, oracle_transfer, rel_err, sample_rows, values)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.fixture(autouse=True)
+def _auto_path():
+    fb.flora_debug_force_path(0)
+    yield
+    fb.flora_debug_force_path(0)
+    torch.cuda.synchronize()
+    assert fb.flora_device_status() == 0
+
+
+def _g(n, m, dtype, seed, var=1e-2):
+    return wl.gaussian_matrix(n, m, var, dtype, seed).to(DEV)
+
+
+# --------------------------------------------------------------------------------------- generator
+@pytest.mark.parametrize("seed,r,m", [(42, 8, 512), (0, 1, 1), (2 ** 64 - 1, 3, 7), (0x123456789ABCDEF0, 32, 770),
+                                      (7, 256, 1030), (99, 64, 4097)])
+def test_generated_projection_is_bit_exact(seed, r, m):
+    ref = orc.materialize_A(seed, r, m)
+    out = torch.full((r, m + 5), 7.0, device=DEV, dtype=torch.float32)
+    fb.flora_materialize_A(out[:, :m], seed)
+    got = out.cpu().numpy()
+    assert np.array_equal(got[:, :m].view(np.uint32), ref.view(np.uint32))
+    assert np.all(got[:, m:] == 7.0)
+    outb = torch.zeros((r, m), device=DEV, dtype=torch.bfloat16)
+    fb.flora_materialize_A(outb, seed)
+    assert np.array_equal(wl.as_numpy(outb), orc.round_to_bf16(ref)[1])
+
+
+# --------------------------------------------------------------------------------------- contractions
+SHAPES = [(1, 1, 1), (5, 7, 3), (33, 100, 8), (130, 257, 17), (64, 512, 32), (300, 1000, 64), (129, 200, 256)]
+
+
+@pytest.mark.parametrize("force_simt", [0, 1])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("n,m,r", SHAPES)
+def test_compress_and_momentum(n, m, r, dtype, force_simt):
+    fb.flora_debug_force_path(force_simt)
+    G = _g(n, m, dtype, 1)
+    S0 = torch.randn(n, r, device=DEV)
+    C = S0.clone()
+    fb.flora_compress_accumulate(G, C, 1234, r)
+    assert rel_err(C.cpu().numpy(), oracle_compress(G, S0, 1234)) <= TOL[dtype]
+    M = S0.clone()
+    fb.flora_momentum_step(G, M, 0.9, 77)
+    assert rel_err(M.cpu().numpy(), oracle_compress(G, S0, 77, a=1.0 - float(np.float32(0.9)), b=0.9)) <= TOL[dtype]
+    # beta = 1 leaves the state alone; beta = 0 ignores what was there (even NaN)
+    M = S0.clone()
+    fb.flora_momentum_step(G, M, 1.0, 77)
+    assert rel_err(M.cpu().numpy(), S0.cpu().numpy()) <= 1e-6
+    M = torch.full((n, r), float("nan"), device=DEV)
+    fb.flora_momentum_step(G, M, 0.0, 77)
+    assert rel_err(M.cpu().numpy(), oracle_compress(G, torch.zeros(n, r), 77)) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("force_simt", [0, 1])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("n,m,r", SHAPES)
+def test_decompress_apply(n, m, r, dtype, force_simt):
+    fb.flora_debug_force_path(force_simt)
+    W0 = _g(n, m, dtype, 2, var=4e-4)
+    C = torch.randn(n, r, device=DEV)
+    W = W0.clone()
+    lr, scale = 0.5, 0.25                       # the update is as large as W: rounding of W does not hide it
+    fb.flora_decompress_apply(W, C, 555, lr, scale)
+    ref = oracle_decompress(W0, C, 555, lr, scale)
+    assert rel_err(values(wl.as_numpy(W)), values(ref)) <= TOL[dtype]
+    w0 = values(wl.as_numpy(W0)).astype(np.float64)
+    assert rel_err(values(wl.as_numpy(W)) - w0, values(ref) - w0) <= TOL[dtype]
+    W = W0.clone()
+    fb.flora_decompress_apply(W, C, 555, 0.0, 1.0)          # lr = 0: bit-identical weights
+    assert torch.equal(W, W0)
+
+
+@pytest.mark.parametrize("operand", ["f32", "bf16"])
+@pytest.mark.parametrize("n,m,r", [(1, 1, 1), (9, 33, 4), (100, 515, 32), (257, 1024, 64), (40, 300, 256)])
+def test_transfer(n, m, r, operand):
+    M0 = torch.randn(n, r, device=DEV)
+    M = M0.clone()
+    fb.flora_resample_transfer(M, m, operand, 10, 11)
+    assert rel_err(M.cpu().numpy(), oracle_transfer(M0, M0, m, operand, 10, 11, 1.0, 0.0)) <= TOL[operand]
+    src = torch.randn(n, r, device=DEV)
+    dst = M0.clone()
+    fb.flora_transfer_axpby(dst, src, m, operand, 3, 4, 0.0125, 0.9)
+    assert rel_err(dst.cpu().numpy(), oracle_transfer(M0, src, m, operand, 3, 4, 0.0125, 0.9)) <= TOL[operand]
+
+
+def test_strided_views_are_honoured():
+    n, m, r = 70, 200, 16
+    Gbig = _g(n, m + 24, "bf16", 3)
+    Cbig = torch.zeros(n, r + 8, device=DEV)
+    fb.flora_compress_accumulate(Gbig[:, :m], Cbig[:, :r], 9, r)
+    ref = oracle_compress(Gbig[:, :m].contiguous(), torch.zeros(n, r), 9)
+    assert rel_err(Cbig[:, :r].cpu().numpy(), ref) <= TOL["bf16"]
+    assert torch.all(Cbig[:, r:] == 0)
+    Wbig = _g(n, m + 24, "bf16", 4)
+    W0 = Wbig.clone()
+    fb.flora_decompress_apply(Wbig[:, :m], Cbig[:, :r], 9, 1.0, 1.0)
+    refw = oracle_decompress(W0[:, :m].contiguous(), Cbig[:, :r].contiguous(), 9, 1.0, 1.0)
+    assert rel_err(values(wl.as_numpy(Wbig[:, :m].contiguous())), values(refw)) <= TOL["bf16"]
+    assert torch.equal(Wbig[:, m:], W0[:, m:])
+
+
+def test_empty_inputs():
+    z = torch.zeros(0, 16, device=DEV)
+    fb.flora_compress_accumulate(z, torch.zeros(0, 4, device=DEV), 1, 4)
+    C = torch.ones(8, 4, device=DEV)
+    fb.flora_compress_accumulate(torch.zeros(8, 0, device=DEV), C, 1, 4)
+    assert torch.all(C == 1)
+    fb.flora_decompress_apply(torch.zeros(8, 0, device=DEV), C, 1, 1.0, 1.0)
+    fb.flora_resample_transfer(torch.zeros(0, 4, device=DEV), 16, "f32", 1, 2)
+    M = torch.ones(3, 4, device=DEV)
+    fb.flora_resample_transfer(M, 0, "f32", 1, 2)              # A has no columns: A A'^T = 0
+    assert torch.all(M == 0)
+
+
+# --------------------------------------------------------------------------------------- configs
+def test_config_single_f32_accumulation_cycle():
+    w = wl.WORKLOADS["single_f32_512"]
+    n, m = w.shapes[0]
+    seedA = 42
+    C = torch.zeros(n, w.r, device=DEV)
+    Cref = np.zeros((n, w.r), dtype=np.float32)
+    A = orc.projection(seedA, w.r, m, "f32")
+    for i in range(w.tau):
+        G = wl.gradient(w, 0, i)
+        fb.flora_compress_accumulate(G.to(DEV), C, seedA, w.r)
+        orc.compress_accumulate(wl.as_numpy(G), A, Cref)
+    assert rel_err(C.cpu().numpy(), Cref) <= TOL["f32"]
+    W0 = wl.weight(w, 0)
+    W = W0.to(DEV)
+    fb.flora_decompress_apply(W, C, seedA, w.lr, 1.0 / w.tau)
+    Wref = wl.as_numpy(W0).copy()
+    orc.decompress_apply(Wref, Cref, A, w.lr, 1.0 / w.tau)
+    assert rel_err(W.cpu().numpy(), Wref) <= TOL["f32"]
+    assert rel_err(W.cpu().numpy() - wl.as_numpy(W0), Wref - wl.as_numpy(W0)) <= TOL["f32"]
+
+
+def _small_set(dtype, r, shapes):
+    G = [_g(n, m, dtype, 100 + i, var=1e-3) for i, (n, m) in enumerate(shapes)]
+    W = [_g(n, m, dtype, 200 + i, var=4e-4) for i, (n, m) in enumerate(shapes)]
+    S = [torch.zeros(n, r, device=DEV) for n, _ in shapes]
+    return G, W, S
+
+
+@pytest.mark.parametrize("force_simt", [0, 1])
+def test_set_accumulation_cycle_and_momentum(force_simt):
+    fb.flora_debug_force_path(force_simt)
+    shapes = [(96, 288), (96, 96), (96, 384), (384, 96), (130, 200)]
+    r, tau = 32, 3
+    G, W, S = _small_set("bf16", r, shapes)
+    W0 = [w.clone() for w in W]
+    fset = fb.FloraSet(G, W, S)
+    seeds = [fb.flora_derive_seed(1, i, 0) for i in range(len(shapes))]
+    Sref = [np.zeros((n, r), dtype=np.float32) for n, _ in shapes]
+    for step in range(tau):
+        Gs = [_g(n, m, "bf16", 1000 * step + i, var=1e-3) for i, (n, m) in enumerate(shapes)]
+        fset.rebind_gradients(Gs)
+        fset.compress_accumulate(seeds)
+        for i in range(len(shapes)):
+            Sref[i] = oracle_compress(Gs[i], torch.from_numpy(Sref[i]), seeds[i])
+    for i in range(len(shapes)):
+        assert rel_err(S[i].cpu().numpy(), Sref[i]) <= TOL["bf16"], i
+    fset.decompress_apply(seeds, 30.0, 1.0 / tau)
+    for i in range(len(shapes)):
+        ref = oracle_decompress(W0[i], S[i], seeds[i], 30.0, 1.0 / tau)
+        assert rel_err(values(wl.as_numpy(W[i])), values(ref)) <= TOL["bf16"], i
+    # momentum with a transfer
+    new = [fb.flora_derive_seed(1, i, 1) for i in range(len(shapes))]
+    Sbefore = [s.clone() for s in S]
+    fset.resample_transfer(seeds, new)
+    for i, (n, m) in enumerate(shapes):
+        assert rel_err(S[i].cpu().numpy(), oracle_transfer(Sbefore[i], Sbefore[i], m, "bf16", seeds[i], new[i], 1.0, 0.0)) <= TOL["bf16"]
+    Sbefore = [s.clone() for s in S]
+    fset.momentum_step(0.9, new)
+    for i in range(len(shapes)):
+        assert rel_err(S[i].cpu().numpy(), oracle_compress(fset.G[i], Sbefore[i], new[i], a=1.0 - float(np.float32(0.9)), b=0.9)) <= TOL["bf16"]
+    fset.zero_state()
+    assert all(torch.all(s == 0) for s in S)
+    fset.close()
+
+
+def test_host_to_device_entry_points():
+    shapes = [(64, 160), (40, 72)]
+    r = 8
+    G, W, S = _small_set("bf16", r, shapes)
+    fset = fb.FloraSet(G, W, S)
+    hostG = [wl.gaussian_matrix(n, m, 1e-3, "bf16", 50 + i).pin_memory() for i, (n, m) in enumerate(shapes)]
+    seeds = [5, 6]
+    fset.compress_accumulate_from_host(hostG, seeds)
+    torch.cuda.synchronize()
+    for i in range(2):
+        assert torch.equal(G[i].cpu(), hostG[i])
+        assert rel_err(S[i].cpu().numpy(), oracle_compress(hostG[i], torch.zeros(shapes[i][0], r), seeds[i])) <= TOL["bf16"]
+    hostW = [torch.empty(n, m, dtype=torch.bfloat16).pin_memory() for n, m in shapes]
+    fset.read_weights_to_host(hostW)
+    torch.cuda.synchronize()
+    assert all(torch.equal(hostW[i], W[i].cpu()) for i in range(2))
+    fset.close()
+
+
+# --------------------------------------------------------------------------------------- full-size configs, sampled rows
+@pytest.mark.parametrize("name", ["gpt2_small_set"])
+def test_full_size_set_sampled_rows(name):
+    w = wl.WORKLOADS[name]
+    count = len(w.shapes)
+    G = [wl.gradient(w, i, 0, device=DEV) for i in range(count)]
+    W = [wl.weight(w, i, device=DEV, std=0.02) for i in range(count)]
+    W0 = [x.clone() for x in W]
+    S = [torch.zeros(n, w.r, device=DEV) for n, _ in w.shapes]
+    fset = fb.FloraSet(G, W, S)
+    seeds = [fb.flora_derive_seed(3, i, 0) for i in range(count)]
+    fset.compress_accumulate(seeds)
+    fset.compress_accumulate(seeds)
+    fset.decompress_apply(seeds, 4.0, 0.5)
+    torch.cuda.synchronize()
+    for i in range(0, count, 5):
+        n, m = w.shapes[i]
+        rows = sample_rows(n, 24, i)
+        Gr = G[i][torch.from_numpy(rows).to(DEV)].cpu()
+        c1 = oracle_compress(Gr, torch.zeros(len(rows), w.r), seeds[i])
+        c2 = oracle_compress(Gr, torch.from_numpy(c1), seeds[i])
+        got = S[i].cpu().numpy()[rows]
+        assert rel_err(got, c2) <= TOL["bf16"], i
+        ref = oracle_decompress(W0[i][torch.from_numpy(rows).to(DEV)].cpu(), torch.from_numpy(got), seeds[i], 4.0, 0.5)
+        assert rel_err(values(wl.as_numpy(W[i])[rows]), values(ref)) <= TOL["bf16"], i
+    fset.close()
