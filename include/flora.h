@@ -121,8 +121,10 @@ typedef struct flora_set flora_set;
 flora_status flora_set_create(int count, const flora_mat* G, const flora_mat* W, const flora_mat* S, flora_set** out);
 flora_status flora_set_destroy(flora_set* set);
 
-/* Re-point the gradient matrices of a set (same shapes, dtypes and leading dimensions).  */
-flora_status flora_set_rebind_gradients(flora_set* set, const flora_mat* G);
+/* Re-point the gradient matrices of a set (same shapes, dtypes and leading dimensions).  The update of
+ * the device-side descriptors is enqueued on `stream`: it is ordered after the set's earlier launches on
+ * that stream and before its later ones.  */
+flora_status flora_set_rebind_gradients(flora_set* set, const flora_mat* G, void* stream);
 
 /* seeds: host array of `count` 64-bit seeds, one per matrix (copied before the call returns). */
 flora_status flora_set_compress_accumulate(flora_set* set, const uint64_t* seeds, void* stream);

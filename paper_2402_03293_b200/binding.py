@@ -65,7 +65,7 @@ def load() -> ctypes.CDLL:
             "flora_materialize_A": (I32, [MP, U64, P]),
             "flora_set_create": (I32, [ctypes.c_int, MP, MP, MP, ctypes.POINTER(P)]),
             "flora_set_destroy": (I32, [P]),
-            "flora_set_rebind_gradients": (I32, [P, MP]),
+            "flora_set_rebind_gradients": (I32, [P, MP, P]),
             "flora_set_compress_accumulate": (I32, [P, ctypes.POINTER(U64), P]),
             "flora_set_momentum_step": (I32, [P, F, ctypes.POINTER(U64), P]),
             "flora_set_decompress_apply": (I32, [P, ctypes.POINTER(U64), F, F, P]),
@@ -232,8 +232,8 @@ class FloraSet:
         except Exception:
             pass
 
-    def rebind_gradients(self, G: List[torch.Tensor]) -> None:
-        _check(load().flora_set_rebind_gradients(self._h, _mat_array(G)), "flora_set_rebind_gradients")
+    def rebind_gradients(self, G: List[torch.Tensor], stream=None) -> None:
+        _check(load().flora_set_rebind_gradients(self._h, _mat_array(G), _stream(stream)), "flora_set_rebind_gradients")
         self.G = G
 
     def compress_accumulate(self, seeds: Sequence[int], stream=None) -> None:

@@ -140,10 +140,13 @@ flora_status transfer_with_scratch(flora_mat* dst, const flora_mat* src, int64_t
     return simt_apply_gram(dst, src, T, a, b, st);
 }
 
-bool use_tc(const flora_mat* big, const flora_mat* sketch)
+bool use_tc_compress(const flora_mat* big, const flora_mat* sketch)
 {
-    if (g_force_path.load(std::memory_order_relaxed) == 1) return false;
-    return tc_supported(big, sketch);
+    return g_force_path.load(std::memory_order_relaxed) != 1 && tc_compress_supported(big, sketch);
+}
+bool use_tc_decompress(const flora_mat* big, const flora_mat* sketch)
+{
+    return g_force_path.load(std::memory_order_relaxed) != 1 && tc_decompress_supported(big, sketch);
 }
 
 }  // namespace
@@ -166,7 +169,7 @@ flora_status flora_compress_accumulate(const flora_mat* G, flora_mat* C, uint64_
     if (st) return st;
     if (r != C->cols) return FLORA_ERR_RANK;
     if (G->rows == 0 || G->cols == 0) return FLORA_OK;
-    if (use_tc(G, C)) return tc_compress_single(G, C, seed, 1.0f, 1.0f, as_stream(stream), g_launches);
+    if (use_tc_compress(G, C)) return tc_compress_single(G, C, seed, 1.0f, 1.0f, as_stream(stream), g_launches);
     return simt_compress(G, C, seed, 1.0f, 1.0f, as_stream(stream));
 }
 
@@ -175,7 +178,7 @@ flora_status flora_momentum_step(const flora_mat* G, flora_mat* M, float beta, u
     flora_status st = check_pair(G, M);
     if (st) return st;
     if (G->rows == 0) return FLORA_OK;
-    if (G->cols > 0 && use_tc(G, M)) return tc_compress_single(G, M, seed, 1.0f - beta, beta, as_stream(stream), g_launches);
+    if (G->cols > 0 && use_tc_compress(G, M)) return tc_compress_single(G, M, seed, 1.0f - beta, beta, as_stream(stream), g_launches);
     return simt_compress(G, M, seed, 1.0f - beta, beta, as_stream(stream));
 }
 
@@ -184,7 +187,7 @@ flora_status flora_decompress_apply(flora_mat* W, const flora_mat* C, uint64_t s
     flora_status st = check_pair(W, C);
     if (st) return st;
     if (W->rows == 0 || W->cols == 0) return FLORA_OK;
-    if (use_tc(W, C)) return tc_decompress_single(W, C, seed, lr * scale, as_stream(stream), g_launches);
+    if (use_tc_decompress(W, C)) return tc_decompress_single(W, C, seed, lr * scale, as_stream(stream), g_launches);
     return simt_decompress(W, C, seed, lr * scale, as_stream(stream));
 }
 
@@ -276,7 +279,7 @@ flora_status flora_set_destroy(flora_set* set)
     return FLORA_OK;
 }
 
-flora_status flora_set_rebind_gradients(flora_set* set, const flora_mat* G)
+flora_status flora_set_rebind_gradients(flora_set* set, const flora_mat* G, void* stream)
 {
     if (!set || !G) return FLORA_ERR_NULL;
     if (!set->has_G) return FLORA_ERR_UNSUPPORTED;
@@ -287,7 +290,7 @@ flora_status flora_set_rebind_gradients(flora_set* set, const flora_mat* G)
         if (G[i].dtype != set->G[i].dtype) return FLORA_ERR_DTYPE;
     }
     std::vector<flora_mat> newG(G, G + set->G.size());
-    flora_status st = tc_set_rebind(set->tc, newG, set->S);
+    flora_status st = tc_set_rebind(set->tc, newG, as_stream(stream));
     if (st) return st;
     set->G.swap(newG);
     return FLORA_OK;

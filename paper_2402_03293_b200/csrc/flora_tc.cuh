@@ -1,27 +1,561 @@
-// Tensor-core (tcgen05) kernels of the path: placeholder interface, nothing eligible yet.
+// Tensor-core kernels of the path for bf16 matrices (sm_100a: TMA, tcgen05.mma, tensor memory).
+//
+//   compress_tc_kernel     S <- b S + a G A^T     (Algorithm 1 compression; Algorithm 2 update of M)
+//   decompress_tc_kernel   W <- W - step * S A    (Algorithm 1 decompression fused with the update)
+//
+// The projection A is generated inside the kernels, tile by tile, straight into the shared-memory
+// layout the tensor core reads (K-major, 128-byte swizzle); it never exists in global memory.
 #pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <algorithm>
 #include <atomic>
 #include <vector>
 
 #include "../../include/flora.h"
+#include "flora_ptx.cuh"
+#include "flora_rng.cuh"
 
 namespace flora {
 
+// ------------------------------------------------------------------------------------------------
+// device-side tables
+// ------------------------------------------------------------------------------------------------
+struct alignas(128) TcMatrix {
+    CUtensorMap map_g;   // gradient G, box 64 columns x 128 rows, 128-byte swizzle
+    CUtensorMap map_w;   // weight W, same box (loads and stores)
+    float* S;            // sketch, n x r fp32
+    int64_t lds;
+    int32_t n, m;
+    int32_t pad[10];
+};
+
+struct K1Item {          // one CTA of the compression kernel
+    int32_t mat;         // index into the matrix table
+    int32_t row0;        // first row of G / S
+    int32_t tiles;       // 128-row tiles handled (1..T)
+    int32_t kstep0;      // first 64-column step
+    int32_t ksteps;      // number of 64-column steps
+    int32_t direct;      // 1: the item covers all columns and owns its rows of S (plain read-modify-write)
+                         // 0: several items add into the same rows (atomic adds; S pre-scaled by b)
+};
+
+struct K2Item {          // one CTA of the decompression kernel
+    int32_t mat;
+    int32_t col0;        // first column of the slab (multiple of 128)
+    int32_t row0;        // first row
+    int32_t tiles;       // 128-row tiles handled
+};
+
+constexpr int SEEDS_PER_LAUNCH = 448;
+struct SeedTable {
+    uint64_t s[SEEDS_PER_LAUNCH];
+};
+
+// ------------------------------------------------------------------------------------------------
+// compression:  S <- b S + a G A^T
+//
+// One CTA handles `tiles` (<= T) 128-row tiles of one matrix over `ksteps` steps of 64 columns.
+// Per step: the producer thread TMA-loads the G tiles; the generator warps write the matching
+// r x 64 tile of A (bf16) into shared memory; one thread issues tiles x 4 MMAs (128 x r_pad x 16)
+// that accumulate in tensor memory.  At the end four warps read the accumulators back and update S.
+// ------------------------------------------------------------------------------------------------
+constexpr int K1_GEN_WARPS = 8;
+constexpr int K1_THREADS = 64 + 32 * K1_GEN_WARPS;
+constexpr int G_TILE_BYTES = 128 * 128;   // 128 rows x 64 bf16
+
+struct K1Smem {                            // barriers and scalars, placed after the tile ring
+    uint64_t full_g[8], full_a[8], empty[8], acc_full;
+    uint32_t tmem_base;
+    int abort;
+};
+
+__device__ __forceinline__ void k1_epilogue_row(float* srow, const uint32_t (&v)[16], int j0, int r, float a, float b,
+                                                bool direct, bool vec_ok)
+{
+    if (vec_ok && j0 + 16 <= r) {
+#pragma unroll
+        for (int u = 0; u < 16; u += 4) {
+            float4* p = reinterpret_cast<float4*>(srow + j0 + u);
+            const float x0 = a * __uint_as_float(v[u]), x1 = a * __uint_as_float(v[u + 1]);
+            const float x2 = a * __uint_as_float(v[u + 2]), x3 = a * __uint_as_float(v[u + 3]);
+            if (!direct) {
+                ptx::red_add_v4(srow + j0 + u, x0, x1, x2, x3);
+            } else if (b == 0.0f) {
+                *p = make_float4(x0, x1, x2, x3);
+            } else {
+                const float4 o = *p;
+                *p = make_float4(fmaf(b, o.x, x0), fmaf(b, o.y, x1), fmaf(b, o.z, x2), fmaf(b, o.w, x3));
+            }
+        }
+    } else {
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+            if (j0 + u < r) {
+                const float x = a * __uint_as_float(v[u]);
+                float* p = srow + j0 + u;
+                if (!direct) atomicAdd(p, x);
+                else *p = (b == 0.0f) ? x : fmaf(b, *p, x);
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(K1_THREADS, 1)
+compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__ items, const __grid_constant__ SeedTable seeds,
+                   int seed_base, int r, float scale, float a, float b, int T, int stages)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
+    const int r_pad = (r + 15) & ~15;
+    const uint32_t a_bytes = (uint32_t)r_pad * 128u;
+    const uint32_t stage_bytes = (uint32_t)T * G_TILE_BYTES + a_bytes;
+    K1Smem* ctl = reinterpret_cast<K1Smem*>(smem_raw + (smem_base - ptx::smem_addr(smem_raw)) + (size_t)stages * stage_bytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    const K1Item item = items[blockIdx.x];
+    const TcMatrix* mat = mats + item.mat;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < T * r_pad) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            ptx::mbar_init(ptx::smem_addr(&ctl->full_g[s]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctl->full_a[s]), K1_GEN_WARPS);
+            ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), 1);
+        }
+        ptx::mbar_init(ptx::smem_addr(&ctl->acc_full), 1);
+        ctl->abort = 0;
+        ptx::fence_barrier_init();
+        ptx::fence_proxy_async_smem();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_addr(&ctl->tmem_base), tmem_cols);
+        ptx::tmem_relinquish();
+    }
+    // rows r .. r_pad of every A tile stay zero for the whole kernel
+    if (r_pad > r) {
+        const int pad_chunks = (r_pad - r) * 8;
+        for (int s = 0; s < stages; ++s)
+            for (int t = threadIdx.x; t < pad_chunks; t += K1_THREADS)
+                ptx::st_shared_v4(smem_base + s * stage_bytes + T * G_TILE_BYTES + (uint32_t)r * 128u + t * 16u, 0, 0, 0, 0);
+        ptx::fence_proxy_async_smem();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = ctl->tmem_base;
+    volatile int* abort = &ctl->abort;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            ptx::prefetch_tensormap(&mat->map_g);
+            int issued = 0;
+            for (int ks = 0; ks < item.ksteps; ++ks) {
+                const int s = ks % stages, it = ks / stages;
+                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort)) break;
+                const uint32_t bar = ptx::smem_addr(&ctl->full_g[s]);
+                ptx::mbar_arrive_expect_tx(bar, (uint32_t)item.tiles * G_TILE_BYTES);
+                for (int t = 0; t < item.tiles; ++t)
+                    ptx::tma_load_2d(smem_base + s * stage_bytes + t * G_TILE_BYTES, &mat->map_g, (item.kstep0 + ks) * 64,
+                                     item.row0 + t * 128, bar);
+                issued = ks + 1;
+            }
+            if (*abort) {
+                // nobody consumes any more: wait (bounded) until the copies still in flight have landed
+                for (int ks = max(0, issued - stages); ks < issued; ++ks)
+                    ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[ks % stages]), (ks / stages) & 1, abort);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = ptx::umma_idesc_bf16((uint32_t)r_pad);
+            bool ok = true;
+            for (int ks = 0; ks < item.ksteps && ok; ++ks) {
+                const int s = ks % stages, it = ks / stages;
+                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[s]), it & 1, abort) &&
+                     ptx::mbar_wait(ptx::smem_addr(&ctl->full_a[s]), it & 1, abort);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t stage = smem_base + s * stage_bytes;
+                const uint32_t a_tile = stage + T * G_TILE_BYTES;
+                for (int t = 0; t < item.tiles; ++t) {
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        ptx::umma_bf16(tmem + t * r_pad, ptx::umma_desc_k_sw128(stage + t * G_TILE_BYTES + kk * 32),
+                                       ptx::umma_desc_k_sw128(a_tile + kk * 32), idesc, (ks | kk) != 0);
+                    }
+                }
+                ptx::umma_commit(ptx::smem_addr(&ctl->empty[s]));
+            }
+            if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->acc_full));
+        }
+    } else {
+        // ------------------------------------------------------------------ generators, then epilogue
+        const int g = threadIdx.x - 64;                       // 0 .. 32*K1_GEN_WARPS-1
+        const PhiloxKey key = make_key(seeds.s[item.mat - seed_base]);
+        const int tasks = r * 8;                              // (row j, 16-byte chunk c) pairs of one A tile
+        bool ok = true;
+        for (int ks = 0; ks < item.ksteps && ok; ++ks) {
+            const int s = ks % stages, it = ks / stages;
+            ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort);
+            if (!ok) break;
+            const uint32_t a_tile = smem_base + s * stage_bytes + T * G_TILE_BYTES;
+            const uint32_t q0 = (uint32_t)(item.kstep0 + ks) * 16u;
+            for (int t = g; t < tasks; t += 32 * K1_GEN_WARPS) {
+                const int j = t >> 3, c = t & 7;
+                const uint2 lo = projection_quad_bf16(q0 + 2 * c, (uint32_t)j, key, scale);
+                const uint2 hi = projection_quad_bf16(q0 + 2 * c + 1, (uint32_t)j, key, scale);
+                ptx::st_shared_v4(a_tile + j * 128 + ((c ^ (j & 7)) << 4), lo.x, lo.y, hi.x, hi.y);
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->full_a[s]));
+        }
+        if (warp < 6 && ok) {
+            // epilogue: warp w reads tensor-memory lanes 32*(w%4) .. +31, i.e. rows of the tile
+            const int quarter = warp & 3;
+            if (ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full), 0, abort)) {
+                ptx::tc_fence_after_sync();
+                const bool vec_ok = ((mat->lds & 3) == 0) && ((reinterpret_cast<uintptr_t>(mat->S) & 15) == 0);
+                for (int t = 0; t < item.tiles; ++t) {
+                    const int64_t row = (int64_t)item.row0 + t * 128 + quarter * 32 + lane;
+                    float* srow = mat->S + row * mat->lds;
+                    for (int j0 = 0; j0 < r_pad; j0 += 16) {
+                        uint32_t v[16];
+                        ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + t * r_pad + j0, v);
+                        ptx::tmem_ld_wait();
+                        if (row < mat->n) k1_epilogue_row(srow, v, j0, r, a, b, item.direct != 0, vec_ok);
+                    }
+                }
+            }
+        }
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem, tmem_cols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
 struct TcSet {
     bool compress_ready = false;
     bool decompress_ready = false;
+    bool transient = false;             // device buffers come from the stream-ordered allocator
+    int count = 0, r = 0;
+    int T = 1, stages = 2;
+    size_t k1_smem = 0;
+    TcMatrix* d_mats = nullptr;
+    K1Item* d_k1 = nullptr;
+    std::vector<TcMatrix> h_mats;
+    std::vector<K1Item> h_k1;
+    std::vector<int> k1_launch_begin;   // item ranges per launch (at most SEEDS_PER_LAUNCH matrices each)
+    std::vector<int> split_mats;        // matrices whose sketch is updated by several items
 };
 
-__device__ int g_flora_error_word;
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-inline bool tc_supported(const flora_mat*, const flora_mat*) { return false; }
-inline flora_status tc_compress_single(const flora_mat*, flora_mat*, uint64_t, float, float, cudaStream_t, std::atomic<uint64_t>&) { return FLORA_ERR_UNSUPPORTED; }
-inline flora_status tc_decompress_single(flora_mat*, const flora_mat*, uint64_t, float, cudaStream_t, std::atomic<uint64_t>&) { return FLORA_ERR_UNSUPPORTED; }
-inline flora_status tc_set_build(TcSet&, const std::vector<flora_mat>&, const std::vector<flora_mat>&, const std::vector<flora_mat>&) { return FLORA_OK; }
-inline void tc_set_free(TcSet&) {}
-inline flora_status tc_set_rebind(TcSet&, const std::vector<flora_mat>&, const std::vector<flora_mat>&) { return FLORA_OK; }
-inline flora_status tc_set_compress(TcSet&, const uint64_t*, float, float, cudaStream_t, std::atomic<uint64_t>&) { return FLORA_ERR_UNSUPPORTED; }
-inline flora_status tc_set_decompress(TcSet&, const uint64_t*, float, cudaStream_t, std::atomic<uint64_t>&) { return FLORA_ERR_UNSUPPORTED; }
+inline EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+// bf16 matrix, box = 64 columns x 128 rows, 128-byte swizzle, zero fill outside the matrix
+inline bool make_map(CUtensorMap* out, const flora_mat& a)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)a.cols, (cuuint64_t)a.rows};
+    cuuint64_t strides[1] = {(cuuint64_t)a.ld * 2};
+    cuuint32_t box[2] = {64, 128};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.data, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline bool tc_mat_ok(const flora_mat& a)
+{
+    return a.dtype == FLORA_BF16 && a.rows >= 128 && a.cols >= 64 && (reinterpret_cast<uintptr_t>(a.data) & 15) == 0 &&
+           (a.ld & 7) == 0 && a.rows < (1ll << 31) - 256 && a.cols < (1ll << 31) - 256;
+}
+
+inline bool tc_compress_supported(const flora_mat* big, const flora_mat* sketch)
+{
+    return tc_mat_ok(*big) && sketch->cols >= 1 && sketch->cols <= 256 && encode_tiled_fn() != nullptr;
+}
+
+inline int sm_count()
+{
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+constexpr size_t SMEM_BUDGET = 216 * 1024;   // per SM, below the 227 KB limit of sm_100
+
+// Tuning knobs (environment variables, read when a set is planned): they change tile shapes and the
+// work split only, never what is computed.
+inline int tune_knob(const char* name, int dflt, int lo, int hi)
+{
+    const char* v = getenv(name);
+    if (!v || !*v) return dflt;
+    return std::max(lo, std::min(hi, atoi(v)));
+}
+
+// Work decomposition of the compression kernel over a set of matrices.
+inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
+{
+    const int r_pad = (r + 15) & ~15;
+    int64_t max_tiles = 1, total_work = 0;       // work unit: one 128-row tile over one 64-column step
+    for (const auto& g : G) {
+        const int64_t tiles = (g.rows + 127) / 128, ks = (g.cols + 63) / 64;
+        max_tiles = std::max(max_tiles, tiles);
+        total_work += tiles * ks;
+    }
+    // T: row tiles per CTA.  More tiles amortise the generation of A (one r x 64 tile serves T x 128 rows);
+    // bounded by tensor memory (T * r_pad <= 512 columns) and by shared memory.  Among the allowed values
+    // take the one that wastes the fewest tile slots over the set, the larger one on a tie.
+    const int t_cap = (int)std::min<int64_t>(std::min<int64_t>(max_tiles, 512 / r_pad), 4);
+    int T = 1;
+    double best = 1e300;
+    for (int cand = t_cap; cand >= 1; --cand) {
+        double padded = 0;
+        for (const auto& g : G) {
+            const int64_t tiles = (g.rows + 127) / 128, ks = (g.cols + 63) / 64;
+            padded += (double)((tiles + cand - 1) / cand * cand) * ks;
+        }
+        if (padded < best * 0.999) {
+            best = padded;
+            T = cand;
+        }
+    }
+    T = tune_knob("FLORA_K1_T", T, 1, 512 / r_pad);
+    const size_t stage = (size_t)T * G_TILE_BYTES + (size_t)r_pad * 128;
+    uint32_t cols = 32;
+    while ((int)cols < T * r_pad) cols <<= 1;
+    // two CTAs per SM when tensor memory allows it and each still gets two stages: the epilogue of one
+    // overlaps the loads of the other
+    int per_sm = (cols <= 256 && 2 * stage <= SMEM_BUDGET / 2) ? 2 : 1;
+    per_sm = tune_knob("FLORA_K1_PER_SM", per_sm, 1, cols <= 256 ? 2 : 1);
+    int stages = (int)std::min<size_t>(8, SMEM_BUDGET / per_sm / stage);
+    stages = tune_knob("FLORA_K1_STAGES", stages, 1, std::max(1, stages));
+    set.T = T;
+    set.stages = stages;
+    set.k1_smem = (size_t)stages * stage + sizeof(K1Smem) + 1024;
+    // column chunks: aim at about `waves` items per CTA slot, at least 8 steps (512 columns) per item
+    const int64_t slots = (int64_t)sm_count() * per_sm;
+    const int waves = tune_knob("FLORA_K1_WAVES", 1, 1, 64);
+    const int64_t target = std::max<int64_t>(8 * T, total_work / (waves * slots) + 1);
+    set.h_k1.clear();
+    set.split_mats.clear();
+    for (size_t i = 0; i < G.size(); ++i) {
+        const auto& g = G[i];
+        if (g.rows == 0 || g.cols == 0) continue;
+        const int64_t tiles = (g.rows + 127) / 128, ks = (g.cols + 63) / 64;
+        int64_t chunk = std::max<int64_t>(8, target / T);
+        int64_t nchunks = (ks + chunk - 1) / chunk;
+        if (nchunks > 1 && ks - (nchunks - 1) * chunk < chunk / 2) --nchunks;    // no short tail item
+        chunk = (ks + nchunks - 1) / nchunks;
+        nchunks = (ks + chunk - 1) / chunk;
+        if (nchunks > 1) set.split_mats.push_back((int)i);
+        for (int64_t t0 = 0; t0 < tiles; t0 += T)
+            for (int64_t c = 0; c < nchunks; ++c) {
+                K1Item it;
+                it.mat = (int)i;
+                it.row0 = (int)(t0 * 128);
+                it.tiles = (int)std::min<int64_t>(T, tiles - t0);
+                it.kstep0 = (int)(c * chunk);
+                it.ksteps = (int)std::min<int64_t>(chunk, ks - c * chunk);
+                it.direct = nchunks == 1;
+                set.h_k1.push_back(it);
+            }
+    }
+    set.k1_launch_begin.clear();
+    int begin_mat = -1;
+    for (size_t k = 0; k < set.h_k1.size(); ++k) {
+        if (begin_mat < 0 || set.h_k1[k].mat >= begin_mat + SEEDS_PER_LAUNCH) {
+            begin_mat = set.h_k1[k].mat;
+            set.k1_launch_begin.push_back((int)k);
+        }
+    }
+    set.k1_launch_begin.push_back((int)set.h_k1.size());
+}
+
+inline void tc_set_free_stream(TcSet& s, cudaStream_t st)
+{
+    if (s.transient) {
+        if (s.d_mats) cudaFreeAsync(s.d_mats, st);
+        if (s.d_k1) cudaFreeAsync(s.d_k1, st);
+    } else {
+        if (s.d_mats) cudaFree(s.d_mats);
+        if (s.d_k1) cudaFree(s.d_k1);
+    }
+    s.d_mats = nullptr;
+    s.d_k1 = nullptr;
+    s.compress_ready = s.decompress_ready = false;
+}
+inline void tc_set_free(TcSet& s) { tc_set_free_stream(s, nullptr); }
+
+template <typename T>
+inline flora_status upload(T** dst, const std::vector<T>& src, bool transient, cudaStream_t st)
+{
+    if (src.empty()) return FLORA_OK;
+    const size_t bytes = src.size() * sizeof(T);
+    if (!*dst) {
+        cudaError_t e = transient ? cudaMallocAsync((void**)dst, bytes, st) : cudaMalloc((void**)dst, bytes);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return FLORA_ERR_ALLOC;
+        }
+    }
+    // pageable source: the runtime stages it before returning, so the vector may change afterwards
+    if (cudaMemcpyAsync(*dst, src.data(), bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return FLORA_ERR_CUDA;
+    return FLORA_OK;
+}
+
+inline flora_status tc_fill_matrices(TcSet& set, const std::vector<flora_mat>& G, const std::vector<flora_mat>& W,
+                                     const std::vector<flora_mat>& S)
+{
+    set.h_mats.assign(S.size(), TcMatrix());
+    for (size_t i = 0; i < S.size(); ++i) {
+        TcMatrix& tm = set.h_mats[i];
+        memset(&tm, 0, sizeof(tm));
+        tm.S = (float*)S[i].data;
+        tm.lds = S[i].ld;
+        const flora_mat& big = !G.empty() ? G[i] : W[i];
+        tm.n = (int32_t)big.rows;
+        tm.m = (int32_t)big.cols;
+        if (!G.empty() && G[i].rows && G[i].cols && !make_map(&tm.map_g, G[i])) return FLORA_ERR_CUDA;
+        if (!W.empty() && W[i].rows && W[i].cols && !make_map(&tm.map_w, W[i])) return FLORA_ERR_CUDA;
+    }
+    return FLORA_OK;
+}
+
+// Builds the tensor-core side of a set; leaves it "not ready" (SIMT kernels are used) if any matrix is not eligible.
+inline flora_status tc_set_build_on(TcSet& set, const std::vector<flora_mat>& G, const std::vector<flora_mat>& W,
+                                    const std::vector<flora_mat>& S, bool transient, cudaStream_t st)
+{
+    set.transient = transient;
+    set.count = (int)S.size();
+    if (S.empty() || !encode_tiled_fn()) return FLORA_OK;
+    set.r = (int)S[0].cols;
+    bool g_ok = !G.empty(), w_ok = false;   // decompression: tensor-core kernel not built yet
+    for (size_t i = 0; i < S.size(); ++i) {
+        if (!G.empty() && !tc_mat_ok(G[i])) g_ok = false;
+        if (!W.empty() && !tc_mat_ok(W[i])) w_ok = false;
+    }
+    if (!g_ok && !w_ok) return FLORA_OK;
+    std::vector<flora_mat> none;
+    flora_status rc = tc_fill_matrices(set, g_ok ? G : none, w_ok ? W : none, S);
+    if (rc) return rc;
+    rc = upload(&set.d_mats, set.h_mats, transient, st);
+    if (rc) return rc;
+    if (g_ok) {
+        plan_compress(set, G, set.r);
+        rc = upload(&set.d_k1, set.h_k1, transient, st);
+        if (rc) return rc;
+        if (cudaFuncSetAttribute(compress_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)set.k1_smem) != cudaSuccess)
+            return FLORA_ERR_CUDA;
+        set.compress_ready = true;
+    }
+    set.decompress_ready = w_ok;
+    return FLORA_OK;
+}
+
+inline flora_status tc_set_build(TcSet& set, const std::vector<flora_mat>& G, const std::vector<flora_mat>& W,
+                                 const std::vector<flora_mat>& S)
+{
+    return tc_set_build_on(set, G, W, S, false, nullptr);
+}
+
+// New gradient pointers, same shapes: only the tensor maps change.
+inline flora_status tc_set_rebind(TcSet& set, const std::vector<flora_mat>& G, cudaStream_t st)
+{
+    if (!set.compress_ready) return FLORA_OK;
+    for (size_t i = 0; i < G.size(); ++i) {
+        if (!tc_mat_ok(G[i])) return FLORA_ERR_ALIGN;
+        if (G[i].rows && G[i].cols && !make_map(&set.h_mats[i].map_g, G[i])) return FLORA_ERR_CUDA;
+    }
+    return upload(&set.d_mats, set.h_mats, false, st);
+}
+
+inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, float b, cudaStream_t st,
+                                    std::atomic<uint64_t>& launches)
+{
+    const int r = set.r;
+    const float scale = 1.0f / sqrtf((float)r);
+    if (b != 1.0f) {
+        // rows updated by several CTAs receive atomic adds: scale them by b first
+        for (int i : set.split_mats) {
+            const TcMatrix& tm = set.h_mats[i];
+            const int64_t total = (int64_t)tm.n * r;
+            scale_rows_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(tm.S, tm.n, r, tm.lds, b);
+            launches.fetch_add(1, std::memory_order_relaxed);
+        }
+    }
+    for (size_t l = 0; l + 1 < set.k1_launch_begin.size(); ++l) {
+        const int begin = set.k1_launch_begin[l], end = set.k1_launch_begin[l + 1];
+        if (end == begin) continue;
+        const int seed_base = set.h_k1[begin].mat;
+        SeedTable table;
+        for (int i = 0; i < SEEDS_PER_LAUNCH; ++i) table.s[i] = seed_base + i < set.count ? seeds[seed_base + i] : 0;
+        compress_tc_kernel<<<end - begin, K1_THREADS, set.k1_smem, st>>>(set.d_mats, set.d_k1 + begin, table, seed_base, r, scale,
+                                                                         a, b, set.T, set.stages);
+        launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    return cudaPeekAtLastError() == cudaSuccess ? FLORA_OK : FLORA_ERR_CUDA;
+}
+
+inline flora_status tc_compress_single(const flora_mat* G, flora_mat* S, uint64_t seed, float a, float b, cudaStream_t st,
+                                       std::atomic<uint64_t>& launches)
+{
+    TcSet set;
+    std::vector<flora_mat> g(1, *G), s(1, *S), none;
+    flora_status rc = tc_set_build_on(set, g, none, s, true, st);
+    if (rc == FLORA_OK) rc = set.compress_ready ? tc_set_compress(set, &seed, a, b, st, launches) : FLORA_ERR_UNSUPPORTED;
+    tc_set_free_stream(set, st);
+    return rc;
+}
+
+inline flora_status tc_decompress_single(flora_mat*, const flora_mat*, uint64_t, float, cudaStream_t, std::atomic<uint64_t>&)
+{
+    return FLORA_ERR_UNSUPPORTED;
+}
+inline flora_status tc_set_decompress(TcSet&, const uint64_t*, float, cudaStream_t, std::atomic<uint64_t>&)
+{
+    return FLORA_ERR_UNSUPPORTED;
+}
+
+inline bool tc_decompress_supported(const flora_mat*, const flora_mat*) { return false; }
+
 inline bool tc_read_and_clear_error(int* word)
 {
     int zero = 0;

@@ -44,7 +44,10 @@ def test_generated_projection_is_bit_exact(seed, r, m):
 
 
 # --------------------------------------------------------------------------------------- contractions
-SHAPES = [(1, 1, 1), (5, 7, 3), (33, 100, 8), (130, 257, 17), (64, 512, 32), (300, 1000, 64), (129, 200, 256)]
+SHAPES = [(1, 1, 1), (5, 7, 3), (33, 100, 8), (130, 257, 17), (64, 512, 32), (300, 1000, 64), (129, 200, 256),
+          # eligible for the tensor-core kernels (bf16, 16-byte aligned rows, n >= 128, m >= 64), ragged tiles and tails
+          (128, 64, 16), (256, 1024, 32), (1000, 2056, 8), (384, 4104, 32), (515, 1288, 128), (200, 776, 96),
+          (700, 1600, 256), (1030, 520, 1)]
 
 
 @pytest.mark.parametrize("force_simt", [0, 1])
@@ -197,6 +200,30 @@ def test_set_accumulation_cycle_and_momentum(force_simt):
         assert rel_err(S[i].cpu().numpy(), oracle_compress(fset.G[i], Sbefore[i], new[i], a=1.0 - float(np.float32(0.9)), b=0.9)) <= TOL["bf16"]
     fset.zero_state()
     assert all(torch.all(s == 0) for s in S)
+    fset.close()
+
+
+def test_set_on_tensor_core_eligible_shapes():
+    shapes = [(256, 576), (384, 128), (128, 1088), (640, 320), (200, 264), (1536, 2048)]
+    r = 32
+    G, W, S = _small_set("bf16", r, shapes)
+    S0 = [torch.randn_like(s) for s in S]
+    for s, s0 in zip(S, S0):
+        s.copy_(s0)
+    fset = fb.FloraSet(G, W, S)
+    seeds = [fb.flora_derive_seed(9, i, 0) for i in range(len(shapes))]
+    fset.compress_accumulate(seeds)
+    for i in range(len(shapes)):
+        assert rel_err(S[i].cpu().numpy(), oracle_compress(G[i], S0[i], seeds[i])) <= TOL["bf16"], i
+    S1 = [s.clone() for s in S]
+    fset.momentum_step(0.5, seeds)
+    for i in range(len(shapes)):
+        assert rel_err(S[i].cpu().numpy(), oracle_compress(G[i], S1[i], seeds[i], a=0.5, b=0.5)) <= TOL["bf16"], i
+    W0 = [w.clone() for w in W]
+    fset.decompress_apply(seeds, 0.01, 1.0)
+    for i in range(len(shapes)):
+        ref = oracle_decompress(W0[i], S[i], seeds[i], 0.01, 1.0)
+        assert rel_err(values(wl.as_numpy(W[i])), values(ref)) <= TOL["bf16"], i
     fset.close()
 
 
