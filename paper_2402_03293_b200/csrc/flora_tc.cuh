@@ -245,6 +245,249 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
 }
 
 // ------------------------------------------------------------------------------------------------
+// decompression fused with the update:  W <- W - step * S A
+//
+// One CTA owns a slab of `bn` (128 or 64) columns of one matrix and `tiles` 128-row tiles of it.
+// It generates the r x bn slab of A once (bf16, as the N x K operand) and then, per row tile:
+// four worker warps convert the fp32 rows of S to the bf16 M x K operand, one thread issues the
+// MMAs (128 x bn x 16 each) into one of two tensor-memory accumulators, the workers combine the
+// accumulator with the W tile that TMA loaded into shared memory, and the producer thread TMA-stores
+// the tile back.  W is read once and written once.
+// ------------------------------------------------------------------------------------------------
+constexpr int K2_THREADS = 192;            // warp 0: TMA loads/stores, warp 1: MMA, warps 2-5: workers
+constexpr int K2_MAX_SLOTS = 6;
+constexpr int W_BOX_BYTES = 128 * 128;     // 128 rows x 64 bf16
+
+struct K2Smem {
+    uint64_t w_full[K2_MAX_SLOTS], out_ready[K2_MAX_SLOTS], a_full, a_empty, acc_full[2], acc_empty[2];
+    uint32_t tmem_base;
+    int abort;
+};
+
+__global__ void __launch_bounds__(K2_THREADS, 1)
+decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict__ items, const __grid_constant__ SeedTable seeds,
+                     int seed_base, int r, float scale, float step, int bn, int slots)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
+    const int k_pad = (r + 63) & ~63;
+    const int kblocks = k_pad >> 6;
+    const int boxes = bn >> 6;                                 // 64-column boxes per W tile
+    const uint32_t slab_block = (uint32_t)bn * 128u;           // one 64-deep K block of the slab
+    const uint32_t slab = smem_base;
+    const uint32_t c_op = slab + kblocks * slab_block;         // 128 x k_pad bf16, K blocks of 16 KB
+    const uint32_t w_ring = c_op + kblocks * (uint32_t)W_BOX_BYTES;
+    const uint32_t slot_bytes = (uint32_t)boxes * W_BOX_BYTES;
+    K2Smem* ctl = reinterpret_cast<K2Smem*>(smem_raw + (w_ring - ptx::smem_addr(smem_raw)) + (size_t)slots * slot_bytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    const K2Item item = items[blockIdx.x];
+    const TcMatrix* mat = mats + item.mat;
+    const uint32_t tmem_cols = 2u * (uint32_t)bn;              // 256 or 128: a power of two >= 32
+    const int live_boxes = min(boxes, (mat->m - item.col0 + 63) >> 6);   // boxes that overlap the matrix
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < slots; ++s) {
+            ptx::mbar_init(ptx::smem_addr(&ctl->w_full[s]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctl->out_ready[s]), 4);
+        }
+        ptx::mbar_init(ptx::smem_addr(&ctl->a_full), 4);
+        ptx::mbar_init(ptx::smem_addr(&ctl->a_empty), 1);
+        for (int s = 0; s < 2; ++s) {
+            ptx::mbar_init(ptx::smem_addr(&ctl->acc_full[s]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[s]), 4);
+        }
+        ctl->abort = 0;
+        ptx::fence_barrier_init();
+        ptx::fence_proxy_async_smem();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_addr(&ctl->tmem_base), tmem_cols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = ctl->tmem_base;
+    volatile int* abort = &ctl->abort;
+
+    // first W tiles are requested before the slab is generated
+    if (warp == 0 && lane == 0) {
+        ptx::prefetch_tensormap(&mat->map_w);
+        for (int i = 0; i < min(slots, item.tiles); ++i) {
+            const uint32_t bar = ptx::smem_addr(&ctl->w_full[i]);
+            ptx::mbar_arrive_expect_tx(bar, (uint32_t)live_boxes * W_BOX_BYTES);
+            for (int bx = 0; bx < live_boxes; ++bx)
+                ptx::tma_load_2d(w_ring + i * slot_bytes + bx * W_BOX_BYTES, &mat->map_w, item.col0 + bx * 64, item.row0 + i * 128, bar);
+        }
+    }
+    {
+        // slab of A as the N x K operand: row = column of W, K = index j of the sketch.  One task makes a
+        // 4-column x 8-j block (eight Philox blocks) and stores one 16-byte chunk per column.
+        const PhiloxKey key = make_key(seeds.s[item.mat - seed_base]);
+        const int jchunks = k_pad >> 3;
+        const int tasks = (bn >> 2) * jchunks;
+        for (int t = threadIdx.x; t < tasks; t += K2_THREADS) {
+            const int jc = t % jchunks, cq = t / jchunks;
+            uint32_t packed[4][4];
+#pragma unroll
+            for (int jj = 0; jj < 8; jj += 2) {
+                float v0[4] = {0.f, 0.f, 0.f, 0.f}, v1[4] = {0.f, 0.f, 0.f, 0.f};
+                const int j = jc * 8 + jj;
+                if (j < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)j, key, scale, v0);
+                if (j + 1 < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)(j + 1), key, scale, v1);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    __nv_bfloat162 pr = __floats2bfloat162_rn(v0[u], v1[u]);
+                    packed[u][jj >> 1] = *reinterpret_cast<uint32_t*>(&pr);
+                }
+            }
+            const uint32_t blk = slab + (jc >> 3) * slab_block;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int c = cq * 4 + u;
+                ptx::st_shared_v4(blk + c * 128 + (((jc & 7) ^ (c & 7)) << 4), packed[u][0], packed[u][1], packed[u][2], packed[u][3]);
+            }
+        }
+        ptx::fence_proxy_async_smem();
+    }
+    __syncthreads();
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA: store finished tiles, refill slots
+        if (lane == 0) {
+            for (int i = 0; i < item.tiles; ++i) {
+                const int s = i % slots;
+                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->out_ready[s]), (i / slots) & 1, abort)) break;
+                for (int bx = 0; bx < live_boxes; ++bx)
+                    ptx::tma_store_2d(&mat->map_w, item.col0 + bx * 64, item.row0 + i * 128, w_ring + s * slot_bytes + bx * W_BOX_BYTES);
+                ptx::tma_store_commit();
+                if (i + slots < item.tiles) {
+                    ptx::tma_store_wait_read<0>();          // the slot has been read out: it can be refilled
+                    const uint32_t bar = ptx::smem_addr(&ctl->w_full[s]);
+                    ptx::mbar_arrive_expect_tx(bar, (uint32_t)live_boxes * W_BOX_BYTES);
+                    for (int bx = 0; bx < live_boxes; ++bx)
+                        ptx::tma_load_2d(w_ring + s * slot_bytes + bx * W_BOX_BYTES, &mat->map_w, item.col0 + bx * 64,
+                                         item.row0 + (i + slots) * 128, bar);
+                }
+            }
+            ptx::tma_store_wait_all<0>();
+            if (*abort) {
+                // loads that nobody consumed: wait (bounded) until they have landed before the CTA exits
+                for (int s = 0; s < min(slots, item.tiles); ++s) {
+                    int last = -1;
+                    for (int i = s; i < item.tiles; i += slots) last = i;
+                    if (last >= 0) ptx::mbar_wait(ptx::smem_addr(&ctl->w_full[s]), (last / slots) & 1, abort);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = ptx::umma_idesc_bf16((uint32_t)bn);
+            const int k16 = (r + 15) >> 4;
+            for (int i = 0; i < item.tiles; ++i) {
+                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->a_full), i & 1, abort)) break;
+                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[i & 1]), ((i >> 1) & 1) ^ 1, abort)) break;
+                ptx::tc_fence_after_sync();
+                for (int k = 0; k < k16; ++k) {
+                    const uint32_t off = (uint32_t)(k & 3) * 32u;
+                    ptx::umma_bf16(tmem + (i & 1) * bn, ptx::umma_desc_k_sw128(c_op + (k >> 2) * W_BOX_BYTES + off),
+                                   ptx::umma_desc_k_sw128(slab + (k >> 2) * slab_block + off), idesc, k != 0);
+                }
+                ptx::umma_commit(ptx::smem_addr(&ctl->a_empty));
+                ptx::umma_commit(ptx::smem_addr(&ctl->acc_full[i & 1]));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ workers: convert S rows, combine with W
+        const int w = threadIdx.x - 64;                        // 0..127
+        const int quarter = warp & 3;                          // tensor-memory lanes 32*quarter .. +31
+        const int jchunks = k_pad >> 3;
+        const bool vec_ok = ((mat->lds & 3) == 0) && ((reinterpret_cast<uintptr_t>(mat->S) & 15) == 0);
+        auto convert = [&](int i) {
+            // rows of S (fp32) -> bf16 operand; consecutive threads take consecutive 8-element pieces of a row
+            for (int t = w; t < 128 * jchunks; t += 128) {
+                const int row = t / jchunks, jc = t % jchunks;
+                const int64_t grow = (int64_t)item.row0 + i * 128 + row;
+                float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                if (grow < mat->n && jc * 8 < r) {
+                    const float* src = mat->S + grow * mat->lds + jc * 8;
+                    if (vec_ok && jc * 8 + 8 <= r) {
+                        const float4 x = *reinterpret_cast<const float4*>(src), y = *reinterpret_cast<const float4*>(src + 4);
+                        v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w; v[4] = y.x; v[5] = y.y; v[6] = y.z; v[7] = y.w;
+                    } else {
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            if (jc * 8 + u < r) v[u] = src[u];
+                    }
+                }
+                uint32_t p[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    __nv_bfloat162 pr = __floats2bfloat162_rn(v[2 * u], v[2 * u + 1]);
+                    p[u] = *reinterpret_cast<uint32_t*>(&pr);
+                }
+                ptx::st_shared_v4(c_op + (jc >> 3) * W_BOX_BYTES + row * 128 + (((jc & 7) ^ (row & 7)) << 4), p[0], p[1], p[2], p[3]);
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->a_full));
+        };
+        convert(0);
+        bool ok = true;
+        for (int i = 0; i < item.tiles && ok; ++i) {
+            if (i + 1 < item.tiles) {
+                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->a_empty), i & 1, abort);
+                if (!ok) break;
+                convert(i + 1);
+            }
+            const int s = i % slots;
+            ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[i & 1]), (i >> 1) & 1, abort) &&
+                 ptx::mbar_wait(ptx::smem_addr(&ctl->w_full[s]), (i / slots) & 1, abort);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            const int row = quarter * 32 + lane;
+            const uint32_t wrow = w_ring + s * slot_bytes + row * 128;
+            for (int c16 = 0; c16 < (live_boxes << 2); ++c16) {
+                uint32_t acc[16];
+                ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + (i & 1) * bn + c16 * 16, acc);
+                ptx::tmem_ld_wait();
+                const uint32_t box = wrow + (c16 >> 2) * W_BOX_BYTES;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t addr = box + (((((c16 & 3) << 1) + h) ^ (row & 7)) << 4);
+                    uint32_t x[4];
+                    ptx::ld_shared_v4(addr, x[0], x[1], x[2], x[3]);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const __nv_bfloat162 old = *reinterpret_cast<__nv_bfloat162*>(&x[u]);
+                        const float lo = fmaf(-step, __uint_as_float(acc[h * 8 + 2 * u]), __low2float(old));
+                        const float hi = fmaf(-step, __uint_as_float(acc[h * 8 + 2 * u + 1]), __high2float(old));
+                        __nv_bfloat162 nw = __floats2bfloat162_rn(lo, hi);
+                        x[u] = *reinterpret_cast<uint32_t*>(&nw);
+                    }
+                    ptx::st_shared_v4(addr, x[0], x[1], x[2], x[3]);
+                }
+            }
+            ptx::tc_fence_before_sync();
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                ptx::mbar_arrive(ptx::smem_addr(&ctl->acc_empty[i & 1]));
+                ptx::mbar_arrive(ptx::smem_addr(&ctl->out_ready[s]));
+            }
+        }
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem, tmem_cols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
 struct TcSet {
@@ -260,6 +503,12 @@ struct TcSet {
     std::vector<K1Item> h_k1;
     std::vector<int> k1_launch_begin;   // item ranges per launch (at most SEEDS_PER_LAUNCH matrices each)
     std::vector<int> split_mats;        // matrices whose sketch is updated by several items
+    // decompression
+    int bn = 128, slots = 2;
+    size_t k2_smem = 0;
+    K2Item* d_k2 = nullptr;
+    std::vector<K2Item> h_k2;
+    std::vector<int> k2_launch_begin;
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -409,17 +658,66 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
     set.k1_launch_begin.push_back((int)set.h_k1.size());
 }
 
+// Work decomposition of the decompression kernel: column slabs of bn columns, cut into runs of row tiles.
+inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
+{
+    const int k_pad = (r + 63) & ~63, kblocks = k_pad / 64;
+    int bn = k_pad > 128 ? 64 : 128;
+    bn = tune_knob("FLORA_K2_BN", bn, 64, 128) >= 128 ? 128 : 64;
+    const size_t fixed = (size_t)kblocks * ((size_t)bn * 128 + W_BOX_BYTES);
+    const size_t slot = (size_t)(bn / 64) * W_BOX_BYTES;
+    // two CTAs per SM when two of them fit (each with at least two W slots): one converts / combines while
+    // the other waits for memory
+    int per_sm = (fixed + 2 * slot + sizeof(K2Smem) + 2048 <= SMEM_BUDGET / 2) ? 2 : 1;
+    per_sm = tune_knob("FLORA_K2_PER_SM", per_sm, 1, 2);
+    int slots = (int)std::min<size_t>(K2_MAX_SLOTS, (SMEM_BUDGET / per_sm - fixed - sizeof(K2Smem) - 2048) / slot);
+    slots = tune_knob("FLORA_K2_SLOTS", slots, 1, std::max(1, slots));
+    set.bn = bn;
+    set.slots = slots;
+    set.k2_smem = fixed + (size_t)slots * slot + sizeof(K2Smem) + 1024;
+    const int run = tune_knob("FLORA_K2_TILES", 16, 1, 1 << 20);      // row tiles per CTA, upper bound
+    set.h_k2.clear();
+    for (size_t i = 0; i < W.size(); ++i) {
+        const auto& w = W[i];
+        if (w.rows == 0 || w.cols == 0) continue;
+        const int64_t rtiles = (w.rows + 127) / 128, slabs = (w.cols + bn - 1) / bn;
+        const int64_t groups = (rtiles + run - 1) / run;
+        const int64_t per = (rtiles + groups - 1) / groups;
+        for (int64_t sl = 0; sl < slabs; ++sl)
+            for (int64_t t0 = 0; t0 < rtiles; t0 += per) {
+                K2Item it;
+                it.mat = (int)i;
+                it.col0 = (int)(sl * bn);
+                it.row0 = (int)(t0 * 128);
+                it.tiles = (int)std::min<int64_t>(per, rtiles - t0);
+                set.h_k2.push_back(it);
+            }
+    }
+    set.k2_launch_begin.clear();
+    int begin_mat = -1;
+    for (size_t k = 0; k < set.h_k2.size(); ++k) {
+        if (begin_mat < 0 || set.h_k2[k].mat >= begin_mat + SEEDS_PER_LAUNCH) {
+            begin_mat = set.h_k2[k].mat;
+            set.k2_launch_begin.push_back((int)k);
+        }
+    }
+    set.k2_launch_begin.push_back((int)set.h_k2.size());
+}
+
 inline void tc_set_free_stream(TcSet& s, cudaStream_t st)
 {
     if (s.transient) {
         if (s.d_mats) cudaFreeAsync(s.d_mats, st);
         if (s.d_k1) cudaFreeAsync(s.d_k1, st);
+        if (s.d_k2) cudaFreeAsync(s.d_k2, st);
     } else {
         if (s.d_mats) cudaFree(s.d_mats);
         if (s.d_k1) cudaFree(s.d_k1);
+        if (s.d_k2) cudaFree(s.d_k2);
     }
     s.d_mats = nullptr;
     s.d_k1 = nullptr;
+    s.d_k2 = nullptr;
     s.compress_ready = s.decompress_ready = false;
 }
 inline void tc_set_free(TcSet& s) { tc_set_free_stream(s, nullptr); }
@@ -467,7 +765,7 @@ inline flora_status tc_set_build_on(TcSet& set, const std::vector<flora_mat>& G,
     set.count = (int)S.size();
     if (S.empty() || !encode_tiled_fn()) return FLORA_OK;
     set.r = (int)S[0].cols;
-    bool g_ok = !G.empty(), w_ok = false;   // decompression: tensor-core kernel not built yet
+    bool g_ok = !G.empty(), w_ok = !W.empty();
     for (size_t i = 0; i < S.size(); ++i) {
         if (!G.empty() && !tc_mat_ok(G[i])) g_ok = false;
         if (!W.empty() && !tc_mat_ok(W[i])) w_ok = false;
@@ -486,7 +784,14 @@ inline flora_status tc_set_build_on(TcSet& set, const std::vector<flora_mat>& G,
             return FLORA_ERR_CUDA;
         set.compress_ready = true;
     }
-    set.decompress_ready = w_ok;
+    if (w_ok) {
+        plan_decompress(set, W, set.r);
+        rc = upload(&set.d_k2, set.h_k2, transient, st);
+        if (rc) return rc;
+        if (cudaFuncSetAttribute(decompress_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)set.k2_smem) != cudaSuccess)
+            return FLORA_ERR_CUDA;
+        set.decompress_ready = true;
+    }
     return FLORA_OK;
 }
 
@@ -545,16 +850,39 @@ inline flora_status tc_compress_single(const flora_mat* G, flora_mat* S, uint64_
     return rc;
 }
 
-inline flora_status tc_decompress_single(flora_mat*, const flora_mat*, uint64_t, float, cudaStream_t, std::atomic<uint64_t>&)
+inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float step, cudaStream_t st,
+                                      std::atomic<uint64_t>& launches)
 {
-    return FLORA_ERR_UNSUPPORTED;
-}
-inline flora_status tc_set_decompress(TcSet&, const uint64_t*, float, cudaStream_t, std::atomic<uint64_t>&)
-{
-    return FLORA_ERR_UNSUPPORTED;
+    const int r = set.r;
+    const float scale = 1.0f / sqrtf((float)r);
+    for (size_t l = 0; l + 1 < set.k2_launch_begin.size(); ++l) {
+        const int begin = set.k2_launch_begin[l], end = set.k2_launch_begin[l + 1];
+        if (end == begin) continue;
+        const int seed_base = set.h_k2[begin].mat;
+        SeedTable table;
+        for (int i = 0; i < SEEDS_PER_LAUNCH; ++i) table.s[i] = seed_base + i < set.count ? seeds[seed_base + i] : 0;
+        decompress_tc_kernel<<<end - begin, K2_THREADS, set.k2_smem, st>>>(set.d_mats, set.d_k2 + begin, table, seed_base, r, scale,
+                                                                           step, set.bn, set.slots);
+        launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    return cudaPeekAtLastError() == cudaSuccess ? FLORA_OK : FLORA_ERR_CUDA;
 }
 
-inline bool tc_decompress_supported(const flora_mat*, const flora_mat*) { return false; }
+inline flora_status tc_decompress_single(flora_mat* W, const flora_mat* S, uint64_t seed, float step, cudaStream_t st,
+                                         std::atomic<uint64_t>& launches)
+{
+    TcSet set;
+    std::vector<flora_mat> w(1, *W), s(1, *S), none;
+    flora_status rc = tc_set_build_on(set, none, w, s, true, st);
+    if (rc == FLORA_OK) rc = set.decompress_ready ? tc_set_decompress(set, &seed, step, st, launches) : FLORA_ERR_UNSUPPORTED;
+    tc_set_free_stream(set, st);
+    return rc;
+}
+
+inline bool tc_decompress_supported(const flora_mat* big, const flora_mat* sketch)
+{
+    return tc_mat_ok(*big) && sketch->cols >= 1 && sketch->cols <= 256 && encode_tiled_fn() != nullptr;
+}
 
 inline bool tc_read_and_clear_error(int* word)
 {
