@@ -358,6 +358,7 @@ flora_status flora_set_resample_transfer(flora_set* set, const uint64_t* seeds_o
 flora_status flora_set_zero_state(flora_set* set, void* stream)
 {
     if (!set) return FLORA_ERR_NULL;
+    if (set->tc.d_mats && g_force_path.load() != 1) return tc_set_zero(set->tc, as_stream(stream), g_launches);
     for (auto& s : set->S) {
         if (s.rows == 0) continue;
         cudaError_t e = cudaMemset2DAsync(s.data, sizeof(float) * s.ld, 0, sizeof(float) * s.cols, (size_t)s.rows, as_stream(stream));

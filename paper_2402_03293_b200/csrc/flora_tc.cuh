@@ -73,22 +73,24 @@ struct K1Smem {                            // barriers and scalars, placed after
     int abort;
 };
 
-__device__ __forceinline__ void k1_epilogue_row(float* srow, const uint32_t (&v)[16], int j0, int r, float a, float b,
-                                                bool direct, bool vec_ok)
+// One row of one tile: sixteen accumulator columns j0..j0+15 into S.  `add_only`: S <- S + a*acc by atomic
+// adds (nothing is read back, so no memory latency sits on the critical path); otherwise the owner of the
+// row computes b*S + a*acc from values `old` that were loaded beforehand.
+__device__ __forceinline__ void k1_store_chunk(float* srow, const uint32_t (&v)[16], const float4 (&old)[4], int j0, int r, float a,
+                                               float b, bool add_only, bool vec_ok)
 {
     if (vec_ok && j0 + 16 <= r) {
 #pragma unroll
         for (int u = 0; u < 16; u += 4) {
-            float4* p = reinterpret_cast<float4*>(srow + j0 + u);
             const float x0 = a * __uint_as_float(v[u]), x1 = a * __uint_as_float(v[u + 1]);
             const float x2 = a * __uint_as_float(v[u + 2]), x3 = a * __uint_as_float(v[u + 3]);
-            if (!direct) {
+            if (add_only) {
                 ptx::red_add_v4(srow + j0 + u, x0, x1, x2, x3);
-            } else if (b == 0.0f) {
-                *p = make_float4(x0, x1, x2, x3);
             } else {
-                const float4 o = *p;
-                *p = make_float4(fmaf(b, o.x, x0), fmaf(b, o.y, x1), fmaf(b, o.z, x2), fmaf(b, o.w, x3));
+                const float4 o = old[u >> 2];
+                *reinterpret_cast<float4*>(srow + j0 + u) =
+                    (b == 0.0f) ? make_float4(x0, x1, x2, x3)
+                                : make_float4(fmaf(b, o.x, x0), fmaf(b, o.y, x1), fmaf(b, o.z, x2), fmaf(b, o.w, x3));
             }
         }
     } else {
@@ -97,7 +99,7 @@ __device__ __forceinline__ void k1_epilogue_row(float* srow, const uint32_t (&v)
             if (j0 + u < r) {
                 const float x = a * __uint_as_float(v[u]);
                 float* p = srow + j0 + u;
-                if (!direct) atomicAdd(p, x);
+                if (add_only) atomicAdd(p, x);
                 else *p = (b == 0.0f) ? x : fmaf(b, *p, x);
             }
         }
@@ -223,14 +225,22 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
             if (ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full), 0, abort)) {
                 ptx::tc_fence_after_sync();
                 const bool vec_ok = ((mat->lds & 3) == 0) && ((reinterpret_cast<uintptr_t>(mat->S) & 15) == 0);
+                // S <- S + a*acc needs no read; a split item adds into rows that were scaled by b beforehand
+                const bool add_only = item.direct == 0 || b == 1.0f;
                 for (int t = 0; t < item.tiles; ++t) {
                     const int64_t row = (int64_t)item.row0 + t * 128 + quarter * 32 + lane;
+                    const bool live = row < mat->n;
                     float* srow = mat->S + row * mat->lds;
                     for (int j0 = 0; j0 < r_pad; j0 += 16) {
+                        float4 old[4] = {};
+                        if (live && !add_only && b != 0.0f && vec_ok && j0 + 16 <= r) {
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) old[u] = *reinterpret_cast<const float4*>(srow + j0 + 4 * u);
+                        }
                         uint32_t v[16];
                         ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + t * r_pad + j0, v);
                         ptx::tmem_ld_wait();
-                        if (row < mat->n) k1_epilogue_row(srow, v, j0, r, a, b, item.direct != 0, vec_ok);
+                        if (live) k1_store_chunk(srow, v, old, j0, r, a, b, add_only, vec_ok);
                     }
                 }
             }
@@ -254,19 +264,19 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
 // accumulator with the W tile that TMA loaded into shared memory, and the producer thread TMA-stores
 // the tile back.  W is read once and written once.
 // ------------------------------------------------------------------------------------------------
-constexpr int K2_THREADS = 192;            // warp 0: TMA loads/stores, warp 1: MMA, warps 2-5: workers
+constexpr int K2_THREADS = 320;            // warp 0: TMA loads/stores, 1: MMA, 2-5: combine with W, 6-9: convert S
 constexpr int K2_MAX_SLOTS = 6;
 constexpr int W_BOX_BYTES = 128 * 128;     // 128 rows x 64 bf16
 
 struct K2Smem {
-    uint64_t w_full[K2_MAX_SLOTS], out_ready[K2_MAX_SLOTS], a_full, a_empty, acc_full[2], acc_empty[2];
+    uint64_t w_full[K2_MAX_SLOTS], out_ready[K2_MAX_SLOTS], a_full[2], a_empty[2], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
     int abort;
 };
 
 __global__ void __launch_bounds__(K2_THREADS, 1)
 decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict__ items, const __grid_constant__ SeedTable seeds,
-                     int seed_base, int r, float scale, float step, int bn, int slots)
+                     int seed_base, int r, float scale, float step, int bn, int slots, int abufs)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
@@ -276,7 +286,8 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
     const uint32_t slab_block = (uint32_t)bn * 128u;           // one 64-deep K block of the slab
     const uint32_t slab = smem_base;
     const uint32_t c_op = slab + kblocks * slab_block;         // 128 x k_pad bf16, K blocks of 16 KB
-    const uint32_t w_ring = c_op + kblocks * (uint32_t)W_BOX_BYTES;
+    const uint32_t c_op_bytes = kblocks * (uint32_t)W_BOX_BYTES;
+    const uint32_t w_ring = c_op + abufs * c_op_bytes;
     const uint32_t slot_bytes = (uint32_t)boxes * W_BOX_BYTES;
     K2Smem* ctl = reinterpret_cast<K2Smem*>(smem_raw + (w_ring - ptx::smem_addr(smem_raw)) + (size_t)slots * slot_bytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -291,9 +302,9 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
             ptx::mbar_init(ptx::smem_addr(&ctl->w_full[s]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->out_ready[s]), 4);
         }
-        ptx::mbar_init(ptx::smem_addr(&ctl->a_full), 4);
-        ptx::mbar_init(ptx::smem_addr(&ctl->a_empty), 1);
         for (int s = 0; s < 2; ++s) {
+            ptx::mbar_init(ptx::smem_addr(&ctl->a_full[s]), 4);
+            ptx::mbar_init(ptx::smem_addr(&ctl->a_empty[s]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->acc_full[s]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[s]), 4);
         }
@@ -387,61 +398,79 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
             const uint32_t idesc = ptx::umma_idesc_bf16((uint32_t)bn);
             const int k16 = (r + 15) >> 4;
             for (int i = 0; i < item.tiles; ++i) {
-                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->a_full), i & 1, abort)) break;
+                const int ab = i % abufs;
+                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->a_full[ab]), (i / abufs) & 1, abort)) break;
                 if (!ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[i & 1]), ((i >> 1) & 1) ^ 1, abort)) break;
                 ptx::tc_fence_after_sync();
                 for (int k = 0; k < k16; ++k) {
                     const uint32_t off = (uint32_t)(k & 3) * 32u;
-                    ptx::umma_bf16(tmem + (i & 1) * bn, ptx::umma_desc_k_sw128(c_op + (k >> 2) * W_BOX_BYTES + off),
+                    ptx::umma_bf16(tmem + (i & 1) * bn, ptx::umma_desc_k_sw128(c_op + ab * c_op_bytes + (k >> 2) * W_BOX_BYTES + off),
                                    ptx::umma_desc_k_sw128(slab + (k >> 2) * slab_block + off), idesc, k != 0);
                 }
-                ptx::umma_commit(ptx::smem_addr(&ctl->a_empty));
+                ptx::umma_commit(ptx::smem_addr(&ctl->a_empty[ab]));
                 ptx::umma_commit(ptx::smem_addr(&ctl->acc_full[i & 1]));
             }
         }
-    } else {
-        // ------------------------------------------------------------------ workers: convert S rows, combine with W
-        const int w = threadIdx.x - 64;                        // 0..127
-        const int quarter = warp & 3;                          // tensor-memory lanes 32*quarter .. +31
+    } else if (warp >= 6) {
+        // ------------------------------------------------------------------ converters: rows of S (fp32) -> bf16 M x K operand
+        // Consecutive threads take consecutive 8-element pieces of a row.  Four pieces per thread are loaded
+        // before any is converted, and the loads of a tile are issued before its buffer is known to be free.
+        const int w = threadIdx.x - 192;                       // 0..127
         const int jchunks = k_pad >> 3;
         const bool vec_ok = ((mat->lds & 3) == 0) && ((reinterpret_cast<uintptr_t>(mat->S) & 15) == 0);
-        auto convert = [&](int i) {
-            // rows of S (fp32) -> bf16 operand; consecutive threads take consecutive 8-element pieces of a row
-            for (int t = w; t < 128 * jchunks; t += 128) {
-                const int row = t / jchunks, jc = t % jchunks;
-                const int64_t grow = (int64_t)item.row0 + i * 128 + row;
-                float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                if (grow < mat->n && jc * 8 < r) {
-                    const float* src = mat->S + grow * mat->lds + jc * 8;
-                    if (vec_ok && jc * 8 + 8 <= r) {
-                        const float4 x = *reinterpret_cast<const float4*>(src), y = *reinterpret_cast<const float4*>(src + 4);
-                        v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w; v[4] = y.x; v[5] = y.y; v[6] = y.z; v[7] = y.w;
-                    } else {
-#pragma unroll
-                        for (int u = 0; u < 8; ++u)
-                            if (jc * 8 + u < r) v[u] = src[u];
-                    }
-                }
-                uint32_t p[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    __nv_bfloat162 pr = __floats2bfloat162_rn(v[2 * u], v[2 * u + 1]);
-                    p[u] = *reinterpret_cast<uint32_t*>(&pr);
-                }
-                ptx::st_shared_v4(c_op + (jc >> 3) * W_BOX_BYTES + row * 128 + (((jc & 7) ^ (row & 7)) << 4), p[0], p[1], p[2], p[3]);
-            }
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->a_full));
-        };
-        convert(0);
         bool ok = true;
         for (int i = 0; i < item.tiles && ok; ++i) {
-            if (i + 1 < item.tiles) {
-                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->a_empty), i & 1, abort);
-                if (!ok) break;
-                convert(i + 1);
+            const int ab = i % abufs;
+            const uint32_t dst = c_op + ab * c_op_bytes;
+            for (int base = 0; base < jchunks && ok; base += 4) {
+                float v[4][8];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int t = w + 128 * (base + u);
+                    const int row = t / jchunks, jc = t % jchunks;
+                    const int64_t grow = (int64_t)item.row0 + i * 128 + row;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) v[u][e] = 0.f;
+                    if (grow < mat->n && jc * 8 < r) {
+                        const float* src = mat->S + grow * mat->lds + jc * 8;
+                        if (vec_ok && jc * 8 + 8 <= r) {
+                            const float4 x = *reinterpret_cast<const float4*>(src), y = *reinterpret_cast<const float4*>(src + 4);
+                            v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
+                            v[u][4] = y.x; v[u][5] = y.y; v[u][6] = y.z; v[u][7] = y.w;
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                if (jc * 8 + e < r) v[u][e] = src[e];
+                        }
+                    }
+                }
+                if (base == 0) {
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->a_empty[ab]), ((i / abufs) & 1) ^ 1, abort);
+                    if (!ok) break;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int t = w + 128 * (base + u);
+                    const int row = t / jchunks, jc = t % jchunks;
+                    uint32_t p[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        __nv_bfloat162 pr = __floats2bfloat162_rn(v[u][2 * e], v[u][2 * e + 1]);
+                        p[e] = *reinterpret_cast<uint32_t*>(&pr);
+                    }
+                    ptx::st_shared_v4(dst + (jc >> 3) * W_BOX_BYTES + row * 128 + (((jc & 7) ^ (row & 7)) << 4), p[0], p[1], p[2], p[3]);
+                }
             }
+            if (!ok) break;
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->a_full[ab]));
+        }
+    } else {
+        // ------------------------------------------------------------------ workers: combine the accumulator with the W tile
+        const int quarter = warp & 3;                          // tensor-memory lanes 32*quarter .. +31
+        bool ok = true;
+        for (int i = 0; i < item.tiles && ok; ++i) {
             const int s = i % slots;
             ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[i & 1]), (i >> 1) & 1, abort) &&
                  ptx::mbar_wait(ptx::smem_addr(&ctl->w_full[s]), (i / slots) & 1, abort);
@@ -487,6 +516,26 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
     }
 }
 
+// S <- b S for the listed matrices (those whose rows receive atomic adds from several CTAs); blockIdx.y = list entry.
+__global__ void scale_sketches_kernel(const TcMatrix* __restrict__ mats, const int* __restrict__ ids, int r, float b)
+{
+    const TcMatrix* mat = mats + ids[blockIdx.y];
+    const int64_t total = (int64_t)mat->n * r;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+        float* p = mat->S + (t / r) * mat->lds + (t % r);
+        *p = (b == 0.0f) ? 0.0f : *p * b;
+    }
+}
+
+// S <- 0 for every matrix of the table (start of an accumulation cycle); blockIdx.y = matrix.
+__global__ void zero_sketches_kernel(const TcMatrix* __restrict__ mats, int r)
+{
+    const TcMatrix* mat = mats + blockIdx.y;
+    const int64_t total = (int64_t)mat->n * r;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x)
+        mat->S[(t / r) * mat->lds + (t % r)] = 0.0f;
+}
+
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
@@ -499,12 +548,13 @@ struct TcSet {
     size_t k1_smem = 0;
     TcMatrix* d_mats = nullptr;
     K1Item* d_k1 = nullptr;
+    int* d_split = nullptr;
     std::vector<TcMatrix> h_mats;
     std::vector<K1Item> h_k1;
     std::vector<int> k1_launch_begin;   // item ranges per launch (at most SEEDS_PER_LAUNCH matrices each)
     std::vector<int> split_mats;        // matrices whose sketch is updated by several items
     // decompression
-    int bn = 128, slots = 2;
+    int bn = 128, slots = 2, abufs = 1;
     size_t k2_smem = 0;
     K2Item* d_k2 = nullptr;
     std::vector<K2Item> h_k2;
@@ -568,7 +618,7 @@ inline int sm_count()
     return n;
 }
 
-constexpr size_t SMEM_BUDGET = 216 * 1024;   // per SM, below the 227 KB limit of sm_100
+constexpr size_t SMEM_BUDGET = 224 * 1024;   // per SM, below the 227 KB limit of sm_100
 
 // Tuning knobs (environment variables, read when a set is planned): they change tile shapes and the
 // work split only, never what is computed.
@@ -664,18 +714,24 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
     const int k_pad = (r + 63) & ~63, kblocks = k_pad / 64;
     int bn = k_pad > 128 ? 64 : 128;
     bn = tune_knob("FLORA_K2_BN", bn, 64, 128) >= 128 ? 128 : 64;
-    const size_t fixed = (size_t)kblocks * ((size_t)bn * 128 + W_BOX_BYTES);
-    const size_t slot = (size_t)(bn / 64) * W_BOX_BYTES;
-    // two CTAs per SM when two of them fit (each with at least two W slots): one converts / combines while
-    // the other waits for memory
-    int per_sm = (fixed + 2 * slot + sizeof(K2Smem) + 2048 <= SMEM_BUDGET / 2) ? 2 : 1;
+    const size_t slab_bytes = (size_t)kblocks * bn * 128, cop = (size_t)kblocks * W_BOX_BYTES;
+    const size_t slot = (size_t)(bn / 64) * W_BOX_BYTES, ctl = sizeof(K2Smem) + 2048;
+    // two CTAs per SM when two of them fit (each with at least two W slots): while one waits for memory the
+    // other converts and combines
+    int per_sm = (slab_bytes + cop + 2 * slot + ctl <= SMEM_BUDGET / 2) ? 2 : 1;
     per_sm = tune_knob("FLORA_K2_PER_SM", per_sm, 1, 2);
-    int slots = (int)std::min<size_t>(K2_MAX_SLOTS, (SMEM_BUDGET / per_sm - fixed - sizeof(K2Smem) - 2048) / slot);
+    const size_t budget = SMEM_BUDGET / per_sm - ctl - slab_bytes;
+    // a second operand buffer lets the conversion run a tile ahead; taken only if two W slots still fit
+    int abufs = (2 * cop + 2 * slot <= budget) ? 2 : 1;
+    abufs = tune_knob("FLORA_K2_ABUFS", abufs, 1, 2);
+    if ((size_t)abufs * cop + slot > budget) abufs = 1;
+    int slots = (int)std::min<size_t>(K2_MAX_SLOTS, (budget - abufs * cop) / slot);
     slots = tune_knob("FLORA_K2_SLOTS", slots, 1, std::max(1, slots));
     set.bn = bn;
     set.slots = slots;
-    set.k2_smem = fixed + (size_t)slots * slot + sizeof(K2Smem) + 1024;
-    const int run = tune_knob("FLORA_K2_TILES", 16, 1, 1 << 20);      // row tiles per CTA, upper bound
+    set.abufs = abufs;
+    set.k2_smem = slab_bytes + abufs * cop + (size_t)slots * slot + sizeof(K2Smem) + 1024;
+    const int run = tune_knob("FLORA_K2_TILES", 8, 1, 1 << 20);      // row tiles per CTA, upper bound
     set.h_k2.clear();
     for (size_t i = 0; i < W.size(); ++i) {
         const auto& w = W[i];
@@ -710,14 +766,17 @@ inline void tc_set_free_stream(TcSet& s, cudaStream_t st)
         if (s.d_mats) cudaFreeAsync(s.d_mats, st);
         if (s.d_k1) cudaFreeAsync(s.d_k1, st);
         if (s.d_k2) cudaFreeAsync(s.d_k2, st);
+        if (s.d_split) cudaFreeAsync(s.d_split, st);
     } else {
         if (s.d_mats) cudaFree(s.d_mats);
         if (s.d_k1) cudaFree(s.d_k1);
         if (s.d_k2) cudaFree(s.d_k2);
+        if (s.d_split) cudaFree(s.d_split);
     }
     s.d_mats = nullptr;
     s.d_k1 = nullptr;
     s.d_k2 = nullptr;
+    s.d_split = nullptr;
     s.compress_ready = s.decompress_ready = false;
 }
 inline void tc_set_free(TcSet& s) { tc_set_free_stream(s, nullptr); }
@@ -780,6 +839,8 @@ inline flora_status tc_set_build_on(TcSet& set, const std::vector<flora_mat>& G,
         plan_compress(set, G, set.r);
         rc = upload(&set.d_k1, set.h_k1, transient, st);
         if (rc) return rc;
+        rc = upload(&set.d_split, set.split_mats, transient, st);
+        if (rc) return rc;
         if (cudaFuncSetAttribute(compress_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)set.k1_smem) != cudaSuccess)
             return FLORA_ERR_CUDA;
         set.compress_ready = true;
@@ -817,12 +878,11 @@ inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, 
 {
     const int r = set.r;
     const float scale = 1.0f / sqrtf((float)r);
-    if (b != 1.0f) {
+    if (b != 1.0f && !set.split_mats.empty()) {
         // rows updated by several CTAs receive atomic adds: scale them by b first
-        for (int i : set.split_mats) {
-            const TcMatrix& tm = set.h_mats[i];
-            const int64_t total = (int64_t)tm.n * r;
-            scale_rows_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(tm.S, tm.n, r, tm.lds, b);
+        for (size_t begin = 0; begin < set.split_mats.size(); begin += 65535) {
+            dim3 grid(16, (unsigned)std::min<size_t>(65535, set.split_mats.size() - begin));
+            scale_sketches_kernel<<<grid, 256, 0, st>>>(set.d_mats, set.d_split + begin, r, b);
             launches.fetch_add(1, std::memory_order_relaxed);
         }
     }
@@ -862,7 +922,7 @@ inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float s
         SeedTable table;
         for (int i = 0; i < SEEDS_PER_LAUNCH; ++i) table.s[i] = seed_base + i < set.count ? seeds[seed_base + i] : 0;
         decompress_tc_kernel<<<end - begin, K2_THREADS, set.k2_smem, st>>>(set.d_mats, set.d_k2 + begin, table, seed_base, r, scale,
-                                                                           step, set.bn, set.slots);
+                                                                           step, set.bn, set.slots, set.abufs);
         launches.fetch_add(1, std::memory_order_relaxed);
     }
     return cudaPeekAtLastError() == cudaSuccess ? FLORA_OK : FLORA_ERR_CUDA;
@@ -882,6 +942,16 @@ inline flora_status tc_decompress_single(flora_mat* W, const flora_mat* S, uint6
 inline bool tc_decompress_supported(const flora_mat* big, const flora_mat* sketch)
 {
     return tc_mat_ok(*big) && sketch->cols >= 1 && sketch->cols <= 256 && encode_tiled_fn() != nullptr;
+}
+
+inline flora_status tc_set_zero(TcSet& set, cudaStream_t st, std::atomic<uint64_t>& launches)
+{
+    for (int begin = 0; begin < set.count; begin += 65535) {
+        dim3 grid(32, (unsigned)std::min(65535, set.count - begin));
+        zero_sketches_kernel<<<grid, 256, 0, st>>>(set.d_mats + begin, set.r);
+        launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    return cudaPeekAtLastError() == cudaSuccess ? FLORA_OK : FLORA_ERR_CUDA;
 }
 
 inline bool tc_read_and_clear_error(int* word)
