@@ -27,10 +27,11 @@ namespace flora {
 struct alignas(128) TcMatrix {
     CUtensorMap map_g;   // gradient G, box 64 columns x 128 rows, 128-byte swizzle
     CUtensorMap map_w;   // weight W, same box (loads and stores)
+    CUtensorMap map_s;   // sketch S (fp32), box 32 columns x 128 rows, 128-byte swizzle
     float* S;            // sketch, n x r fp32
     int64_t lds;
     int32_t n, m;
-    int32_t pad[10];
+    int32_t pad[26];
 };
 
 struct K1Item {          // one CTA of the compression kernel
@@ -258,36 +259,37 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
 // decompression fused with the update:  W <- W - step * S A
 //
 // One CTA owns a slab of `bn` (128 or 64) columns of one matrix and `tiles` 128-row tiles of it.
-// It generates the r x bn slab of A once (bf16, as the N x K operand) and then, per row tile:
-// four worker warps convert the fp32 rows of S to the bf16 M x K operand, one thread issues the
-// MMAs (128 x bn x 16 each) into one of two tensor-memory accumulators, the workers combine the
-// accumulator with the W tile that TMA loaded into shared memory, and the producer thread TMA-stores
-// the tile back.  W is read once and written once.
+// It generates the r x bn slab of A once (the N x K operand: bf16 values held in 32-bit containers)
+// and then streams row tiles: TMA brings the fp32 rows of S in 32-column chunks and the W tile into
+// shared memory; one thread issues tf32 MMAs (128 x bn x 8) that read S as it is stored, into one of
+// two tensor-memory accumulators; four warps combine the accumulator with the W tile in shared memory
+// and a TMA store writes the tile back.  W is read once and written once, S is never converted.
 // ------------------------------------------------------------------------------------------------
-constexpr int K2_THREADS = 320;            // warp 0: TMA loads/stores, 1: MMA, 2-5: combine with W, 6-9: convert S
+constexpr int K2_THREADS = 256;   // warp 0: W loads, 1: MMA, 2-5: combine, 6: S loads, 7: W stores
 constexpr int K2_MAX_SLOTS = 6;
+constexpr int K2_MAX_CSTAGES = 8;
 constexpr int W_BOX_BYTES = 128 * 128;     // 128 rows x 64 bf16
+constexpr int S_CHUNK_BYTES = 128 * 128;   // 128 rows x 32 fp32
 
 struct K2Smem {
-    uint64_t w_full[K2_MAX_SLOTS], out_ready[K2_MAX_SLOTS], a_full[2], a_empty[2], acc_full[2], acc_empty[2];
+    uint64_t w_full[K2_MAX_SLOTS], w_free[K2_MAX_SLOTS], out_ready[K2_MAX_SLOTS];
+    uint64_t c_full[K2_MAX_CSTAGES], c_empty[K2_MAX_CSTAGES], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
     int abort;
 };
 
 __global__ void __launch_bounds__(K2_THREADS, 1)
 decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict__ items, const __grid_constant__ SeedTable seeds,
-                     int seed_base, int r, float scale, float step, int bn, int slots, int abufs)
+                     int seed_base, int r, float scale, float step, int bn, int slots, int cstages)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
-    const int k_pad = (r + 63) & ~63;
-    const int kblocks = k_pad >> 6;
+    const int kchunks = (r + 31) >> 5;                         // 32-deep K chunks (one 128-byte row of fp32 each)
     const int boxes = bn >> 6;                                 // 64-column boxes per W tile
-    const uint32_t slab_block = (uint32_t)bn * 128u;           // one 64-deep K block of the slab
+    const uint32_t slab_block = (uint32_t)bn * 128u;           // one K chunk of the slab
     const uint32_t slab = smem_base;
-    const uint32_t c_op = slab + kblocks * slab_block;         // 128 x k_pad bf16, K blocks of 16 KB
-    const uint32_t c_op_bytes = kblocks * (uint32_t)W_BOX_BYTES;
-    const uint32_t w_ring = c_op + abufs * c_op_bytes;
+    const uint32_t c_ring = slab + kchunks * slab_block;
+    const uint32_t w_ring = c_ring + cstages * (uint32_t)S_CHUNK_BYTES;
     const uint32_t slot_bytes = (uint32_t)boxes * W_BOX_BYTES;
     K2Smem* ctl = reinterpret_cast<K2Smem*>(smem_raw + (w_ring - ptx::smem_addr(smem_raw)) + (size_t)slots * slot_bytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -300,11 +302,14 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
     if (threadIdx.x == 0) {
         for (int s = 0; s < slots; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->w_full[s]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctl->w_free[s]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->out_ready[s]), 4);
         }
+        for (int s = 0; s < cstages; ++s) {
+            ptx::mbar_init(ptx::smem_addr(&ctl->c_full[s]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctl->c_empty[s]), 1);
+        }
         for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(ptx::smem_addr(&ctl->a_full[s]), 4);
-            ptx::mbar_init(ptx::smem_addr(&ctl->a_empty[s]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->acc_full[s]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[s]), 4);
         }
@@ -322,42 +327,51 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
     const uint32_t tmem = ctl->tmem_base;
     volatile int* abort = &ctl->abort;
 
-    // first W tiles are requested before the slab is generated
+    // The first W tiles and S chunks are requested before the slab is generated (fresh slots: nothing to wait for).
+    const int total_chunks = item.tiles * kchunks;
+    auto load_w = [&](int i) {
+        const int s = i % slots;
+        const uint32_t bar = ptx::smem_addr(&ctl->w_full[s]);
+        ptx::mbar_arrive_expect_tx(bar, (uint32_t)live_boxes * W_BOX_BYTES);
+        for (int bx = 0; bx < live_boxes; ++bx)
+            ptx::tma_load_2d(w_ring + s * slot_bytes + bx * W_BOX_BYTES, &mat->map_w, item.col0 + bx * 64, item.row0 + i * 128, bar);
+    };
+    auto load_s = [&](int c) {
+        const int s = c % cstages;
+        const uint32_t bar = ptx::smem_addr(&ctl->c_full[s]);
+        ptx::mbar_arrive_expect_tx(bar, S_CHUNK_BYTES);
+        ptx::tma_load_2d(c_ring + s * S_CHUNK_BYTES, &mat->map_s, (c % kchunks) * 32, item.row0 + (c / kchunks) * 128, bar);
+    };
     if (warp == 0 && lane == 0) {
         ptx::prefetch_tensormap(&mat->map_w);
-        for (int i = 0; i < min(slots, item.tiles); ++i) {
-            const uint32_t bar = ptx::smem_addr(&ctl->w_full[i]);
-            ptx::mbar_arrive_expect_tx(bar, (uint32_t)live_boxes * W_BOX_BYTES);
-            for (int bx = 0; bx < live_boxes; ++bx)
-                ptx::tma_load_2d(w_ring + i * slot_bytes + bx * W_BOX_BYTES, &mat->map_w, item.col0 + bx * 64, item.row0 + i * 128, bar);
-        }
+        for (int i = 0; i < min(slots, item.tiles); ++i) load_w(i);
+    } else if (warp == 6 && lane == 0) {
+        ptx::prefetch_tensormap(&mat->map_s);
+        for (int c = 0; c < min(cstages, total_chunks); ++c) load_s(c);
     }
     {
-        // slab of A as the N x K operand: row = column of W, K = index j of the sketch.  One task makes a
-        // 4-column x 8-j block (eight Philox blocks) and stores one 16-byte chunk per column.
+        // slab of A as the N x K operand: row = column of W, K = index j of the sketch, values rounded to bf16
+        // and widened to 32 bits (exact in tf32).  One task makes a 4-column x 4-j block (four Philox blocks)
+        // and stores one 16-byte chunk per column; j >= r is written as zero.
         const PhiloxKey key = make_key(seeds.s[item.mat - seed_base]);
-        const int jchunks = k_pad >> 3;
-        const int tasks = (bn >> 2) * jchunks;
+        const int jgroups = kchunks * 8;
+        const int tasks = (bn >> 2) * jgroups;
         for (int t = threadIdx.x; t < tasks; t += K2_THREADS) {
-            const int jc = t % jchunks, cq = t / jchunks;
-            uint32_t packed[4][4];
+            const int jg = t % jgroups, cq = t / jgroups;
+            float v[4][4];
 #pragma unroll
-            for (int jj = 0; jj < 8; jj += 2) {
-                float v0[4] = {0.f, 0.f, 0.f, 0.f}, v1[4] = {0.f, 0.f, 0.f, 0.f};
-                const int j = jc * 8 + jj;
-                if (j < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)j, key, scale, v0);
-                if (j + 1 < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)(j + 1), key, scale, v1);
+            for (int jj = 0; jj < 4; ++jj) {
+                float q[4] = {0.f, 0.f, 0.f, 0.f};
+                if (jg * 4 + jj < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)(jg * 4 + jj), key, scale, q);
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    __nv_bfloat162 pr = __floats2bfloat162_rn(v0[u], v1[u]);
-                    packed[u][jj >> 1] = *reinterpret_cast<uint32_t*>(&pr);
-                }
+                for (int u = 0; u < 4; ++u) v[u][jj] = bf16_round(q[u]);
             }
-            const uint32_t blk = slab + (jc >> 3) * slab_block;
+            const uint32_t blk = slab + (jg >> 3) * slab_block;
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int c = cq * 4 + u;
-                ptx::st_shared_v4(blk + c * 128 + (((jc & 7) ^ (c & 7)) << 4), packed[u][0], packed[u][1], packed[u][2], packed[u][3]);
+                ptx::st_shared_v4(blk + c * 128 + (((jg & 7) ^ (c & 7)) << 4), __float_as_uint(v[u][0]), __float_as_uint(v[u][1]),
+                                  __float_as_uint(v[u][2]), __float_as_uint(v[u][3]));
             }
         }
         ptx::fence_proxy_async_smem();
@@ -365,7 +379,54 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
     __syncthreads();
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA: store finished tiles, refill slots
+        // ------------------------------------------------------------------ W tile loads: refill slots as the stores free them
+        if (lane == 0) {
+            int issued = min(slots, item.tiles);
+            for (int i = issued; i < item.tiles; ++i) {
+                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->w_free[i % slots]), ((i / slots) & 1) ^ 1, abort)) break;
+                load_w(i);
+                issued = i + 1;
+            }
+            if (*abort)   // loads that nobody consumed: wait (bounded) until they have landed
+                for (int i = max(0, issued - slots); i < issued; ++i)
+                    ptx::mbar_wait(ptx::smem_addr(&ctl->w_full[i % slots]), (i / slots) & 1, abort);
+        }
+    } else if (warp == 6) {
+        // ------------------------------------------------------------------ S chunk loads (fp32 rows, 32 columns each)
+        if (lane == 0) {
+            int issued = min(cstages, total_chunks);
+            for (int c = issued; c < total_chunks; ++c) {
+                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->c_empty[c % cstages]), ((c / cstages) & 1) ^ 1, abort)) break;
+                load_s(c);
+                issued = c + 1;
+            }
+            if (*abort)
+                for (int c = max(0, issued - cstages); c < issued; ++c)
+                    ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[c % cstages]), (c / cstages) & 1, abort);
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = ptx::umma_idesc_tf32((uint32_t)bn);
+            bool ok = true;
+            for (int i = 0; i < item.tiles && ok; ++i) {
+                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[i & 1]), ((i >> 1) & 1) ^ 1, abort);
+                for (int kc = 0; kc < kchunks && ok; ++kc) {
+                    const int c = i * kchunks + kc, s = c % cstages;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[s]), (c / cstages) & 1, abort);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+#pragma unroll
+                    for (int k8 = 0; k8 < 4; ++k8)
+                        ptx::umma_tf32(tmem + (i & 1) * bn, ptx::umma_desc_k_sw128(c_ring + s * S_CHUNK_BYTES + k8 * 32),
+                                       ptx::umma_desc_k_sw128(slab + kc * slab_block + k8 * 32), idesc, (kc | k8) != 0);
+                    ptx::umma_commit(ptx::smem_addr(&ctl->c_empty[s]));
+                }
+                if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->acc_full[i & 1]));
+            }
+        }
+    } else if (warp == 7) {
+        // ------------------------------------------------------------------ W tile stores
         if (lane == 0) {
             for (int i = 0; i < item.tiles; ++i) {
                 const int s = i % slots;
@@ -373,101 +434,13 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
                 for (int bx = 0; bx < live_boxes; ++bx)
                     ptx::tma_store_2d(&mat->map_w, item.col0 + bx * 64, item.row0 + i * 128, w_ring + s * slot_bytes + bx * W_BOX_BYTES);
                 ptx::tma_store_commit();
-                if (i + slots < item.tiles) {
-                    ptx::tma_store_wait_read<0>();          // the slot has been read out: it can be refilled
-                    const uint32_t bar = ptx::smem_addr(&ctl->w_full[s]);
-                    ptx::mbar_arrive_expect_tx(bar, (uint32_t)live_boxes * W_BOX_BYTES);
-                    for (int bx = 0; bx < live_boxes; ++bx)
-                        ptx::tma_load_2d(w_ring + s * slot_bytes + bx * W_BOX_BYTES, &mat->map_w, item.col0 + bx * 64,
-                                         item.row0 + (i + slots) * 128, bar);
-                }
+                ptx::tma_store_wait_read<0>();              // the slot has been read out: it can be refilled
+                ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[s]));
             }
             ptx::tma_store_wait_all<0>();
-            if (*abort) {
-                // loads that nobody consumed: wait (bounded) until they have landed before the CTA exits
-                for (int s = 0; s < min(slots, item.tiles); ++s) {
-                    int last = -1;
-                    for (int i = s; i < item.tiles; i += slots) last = i;
-                    if (last >= 0) ptx::mbar_wait(ptx::smem_addr(&ctl->w_full[s]), (last / slots) & 1, abort);
-                }
-            }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = ptx::umma_idesc_bf16((uint32_t)bn);
-            const int k16 = (r + 15) >> 4;
-            for (int i = 0; i < item.tiles; ++i) {
-                const int ab = i % abufs;
-                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->a_full[ab]), (i / abufs) & 1, abort)) break;
-                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[i & 1]), ((i >> 1) & 1) ^ 1, abort)) break;
-                ptx::tc_fence_after_sync();
-                for (int k = 0; k < k16; ++k) {
-                    const uint32_t off = (uint32_t)(k & 3) * 32u;
-                    ptx::umma_bf16(tmem + (i & 1) * bn, ptx::umma_desc_k_sw128(c_op + ab * c_op_bytes + (k >> 2) * W_BOX_BYTES + off),
-                                   ptx::umma_desc_k_sw128(slab + (k >> 2) * slab_block + off), idesc, k != 0);
-                }
-                ptx::umma_commit(ptx::smem_addr(&ctl->a_empty[ab]));
-                ptx::umma_commit(ptx::smem_addr(&ctl->acc_full[i & 1]));
-            }
-        }
-    } else if (warp >= 6) {
-        // ------------------------------------------------------------------ converters: rows of S (fp32) -> bf16 M x K operand
-        // Consecutive threads take consecutive 8-element pieces of a row.  Four pieces per thread are loaded
-        // before any is converted, and the loads of a tile are issued before its buffer is known to be free.
-        const int w = threadIdx.x - 192;                       // 0..127
-        const int jchunks = k_pad >> 3;
-        const bool vec_ok = ((mat->lds & 3) == 0) && ((reinterpret_cast<uintptr_t>(mat->S) & 15) == 0);
-        bool ok = true;
-        for (int i = 0; i < item.tiles && ok; ++i) {
-            const int ab = i % abufs;
-            const uint32_t dst = c_op + ab * c_op_bytes;
-            for (int base = 0; base < jchunks && ok; base += 4) {
-                float v[4][8];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int t = w + 128 * (base + u);
-                    const int row = t / jchunks, jc = t % jchunks;
-                    const int64_t grow = (int64_t)item.row0 + i * 128 + row;
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) v[u][e] = 0.f;
-                    if (grow < mat->n && jc * 8 < r) {
-                        const float* src = mat->S + grow * mat->lds + jc * 8;
-                        if (vec_ok && jc * 8 + 8 <= r) {
-                            const float4 x = *reinterpret_cast<const float4*>(src), y = *reinterpret_cast<const float4*>(src + 4);
-                            v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
-                            v[u][4] = y.x; v[u][5] = y.y; v[u][6] = y.z; v[u][7] = y.w;
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < 8; ++e)
-                                if (jc * 8 + e < r) v[u][e] = src[e];
-                        }
-                    }
-                }
-                if (base == 0) {
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->a_empty[ab]), ((i / abufs) & 1) ^ 1, abort);
-                    if (!ok) break;
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int t = w + 128 * (base + u);
-                    const int row = t / jchunks, jc = t % jchunks;
-                    uint32_t p[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        __nv_bfloat162 pr = __floats2bfloat162_rn(v[u][2 * e], v[u][2 * e + 1]);
-                        p[e] = *reinterpret_cast<uint32_t*>(&pr);
-                    }
-                    ptx::st_shared_v4(dst + (jc >> 3) * W_BOX_BYTES + row * 128 + (((jc & 7) ^ (row & 7)) << 4), p[0], p[1], p[2], p[3]);
-                }
-            }
-            if (!ok) break;
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->a_full[ab]));
-        }
-    } else {
-        // ------------------------------------------------------------------ workers: combine the accumulator with the W tile
+    } else if (warp >= 2 && warp <= 5) {
+        // ------------------------------------------------------------------ combine the accumulator with the W tile
         const int quarter = warp & 3;                          // tensor-memory lanes 32*quarter .. +31
         bool ok = true;
         for (int i = 0; i < item.tiles && ok; ++i) {
@@ -554,7 +527,7 @@ struct TcSet {
     std::vector<int> k1_launch_begin;   // item ranges per launch (at most SEEDS_PER_LAUNCH matrices each)
     std::vector<int> split_mats;        // matrices whose sketch is updated by several items
     // decompression
-    int bn = 128, slots = 2, abufs = 1;
+    int bn = 128, slots = 2, cstages = 2;
     size_t k2_smem = 0;
     K2Item* d_k2 = nullptr;
     std::vector<K2Item> h_k2;
@@ -595,6 +568,24 @@ inline bool make_map(CUtensorMap* out, const flora_mat& a)
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 sketch, box = 32 columns x 128 rows, 128-byte swizzle, zero fill outside the matrix
+inline bool make_map_f32(CUtensorMap* out, const flora_mat& a)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)a.cols, (cuuint64_t)a.rows};
+    cuuint64_t strides[1] = {(cuuint64_t)a.ld * 4};
+    cuuint32_t box[2] = {32, 128};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, a.data, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline bool tc_sketch_ok(const flora_mat& s)
+{
+    return (reinterpret_cast<uintptr_t>(s.data) & 15) == 0 && (s.ld & 3) == 0 && s.cols >= 1 && s.cols <= 256;
+}
+
 inline bool tc_mat_ok(const flora_mat& a)
 {
     return a.dtype == FLORA_BF16 && a.rows >= 128 && a.cols >= 64 && (reinterpret_cast<uintptr_t>(a.data) & 15) == 0 &&
@@ -603,7 +594,7 @@ inline bool tc_mat_ok(const flora_mat& a)
 
 inline bool tc_compress_supported(const flora_mat* big, const flora_mat* sketch)
 {
-    return tc_mat_ok(*big) && sketch->cols >= 1 && sketch->cols <= 256 && encode_tiled_fn() != nullptr;
+    return tc_mat_ok(*big) && tc_sketch_ok(*sketch) && encode_tiled_fn() != nullptr;
 }
 
 inline int sm_count()
@@ -711,26 +702,25 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
 // Work decomposition of the decompression kernel: column slabs of bn columns, cut into runs of row tiles.
 inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
 {
-    const int k_pad = (r + 63) & ~63, kblocks = k_pad / 64;
-    int bn = k_pad > 128 ? 64 : 128;
+    const int kchunks = (r + 31) / 32;
+    int bn = kchunks > 4 ? 64 : 128;
     bn = tune_knob("FLORA_K2_BN", bn, 64, 128) >= 128 ? 128 : 64;
-    const size_t slab_bytes = (size_t)kblocks * bn * 128, cop = (size_t)kblocks * W_BOX_BYTES;
-    const size_t slot = (size_t)(bn / 64) * W_BOX_BYTES, ctl = sizeof(K2Smem) + 2048;
-    // two CTAs per SM when two of them fit (each with at least two W slots): while one waits for memory the
-    // other converts and combines
-    int per_sm = (slab_bytes + cop + 2 * slot + ctl <= SMEM_BUDGET / 2) ? 2 : 1;
+    const size_t slab_bytes = (size_t)kchunks * bn * 128, slot = (size_t)(bn / 64) * W_BOX_BYTES, ctl = sizeof(K2Smem) + 1024;
+    // two CTAs per SM when two of them fit (each with two W slots and one S chunk): the fixed cost of one
+    // CTA (its slab) hides behind the streaming of the other
+    const size_t per_cta_max = 113 * 1024;                       // half of an SM's shared memory minus the reserve
+    int per_sm = (slab_bytes + S_CHUNK_BYTES + 2 * slot + ctl <= per_cta_max) ? 2 : 1;
     per_sm = tune_knob("FLORA_K2_PER_SM", per_sm, 1, 2);
-    const size_t budget = SMEM_BUDGET / per_sm - ctl - slab_bytes;
-    // a second operand buffer lets the conversion run a tile ahead; taken only if two W slots still fit
-    int abufs = (2 * cop + 2 * slot <= budget) ? 2 : 1;
-    abufs = tune_knob("FLORA_K2_ABUFS", abufs, 1, 2);
-    if ((size_t)abufs * cop + slot > budget) abufs = 1;
-    int slots = (int)std::min<size_t>(K2_MAX_SLOTS, (budget - abufs * cop) / slot);
+    const size_t budget = (per_sm == 2 ? per_cta_max : SMEM_BUDGET) - ctl - slab_bytes;
+    int cstages = std::max(2, std::min(kchunks + 1, 4));
+    cstages = tune_knob("FLORA_K2_CSTAGES", cstages, 1, K2_MAX_CSTAGES);
+    while (cstages > 1 && (size_t)cstages * S_CHUNK_BYTES + 2 * slot > budget) --cstages;
+    int slots = (int)std::min<size_t>(K2_MAX_SLOTS, (budget - (size_t)cstages * S_CHUNK_BYTES) / slot);
     slots = tune_knob("FLORA_K2_SLOTS", slots, 1, std::max(1, slots));
     set.bn = bn;
     set.slots = slots;
-    set.abufs = abufs;
-    set.k2_smem = slab_bytes + abufs * cop + (size_t)slots * slot + sizeof(K2Smem) + 1024;
+    set.cstages = cstages;
+    set.k2_smem = slab_bytes + (size_t)cstages * S_CHUNK_BYTES + (size_t)slots * slot + sizeof(K2Smem) + 1024;
     const int run = tune_knob("FLORA_K2_TILES", 8, 1, 1 << 20);      // row tiles per CTA, upper bound
     set.h_k2.clear();
     for (size_t i = 0; i < W.size(); ++i) {
@@ -811,7 +801,7 @@ inline flora_status tc_fill_matrices(TcSet& set, const std::vector<flora_mat>& G
         tm.n = (int32_t)big.rows;
         tm.m = (int32_t)big.cols;
         if (!G.empty() && G[i].rows && G[i].cols && !make_map(&tm.map_g, G[i])) return FLORA_ERR_CUDA;
-        if (!W.empty() && W[i].rows && W[i].cols && !make_map(&tm.map_w, W[i])) return FLORA_ERR_CUDA;
+        if (!W.empty() && W[i].rows && W[i].cols && (!make_map(&tm.map_w, W[i]) || !make_map_f32(&tm.map_s, S[i]))) return FLORA_ERR_CUDA;
     }
     return FLORA_OK;
 }
@@ -827,7 +817,7 @@ inline flora_status tc_set_build_on(TcSet& set, const std::vector<flora_mat>& G,
     bool g_ok = !G.empty(), w_ok = !W.empty();
     for (size_t i = 0; i < S.size(); ++i) {
         if (!G.empty() && !tc_mat_ok(G[i])) g_ok = false;
-        if (!W.empty() && !tc_mat_ok(W[i])) w_ok = false;
+        if (!W.empty() && (!tc_mat_ok(W[i]) || !tc_sketch_ok(S[i]))) w_ok = false;
     }
     if (!g_ok && !w_ok) return FLORA_OK;
     std::vector<flora_mat> none;
@@ -922,7 +912,7 @@ inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float s
         SeedTable table;
         for (int i = 0; i < SEEDS_PER_LAUNCH; ++i) table.s[i] = seed_base + i < set.count ? seeds[seed_base + i] : 0;
         decompress_tc_kernel<<<end - begin, K2_THREADS, set.k2_smem, st>>>(set.d_mats, set.d_k2 + begin, table, seed_base, r, scale,
-                                                                           step, set.bn, set.slots, set.abufs);
+                                                                           step, set.bn, set.slots, set.cstages);
         launches.fetch_add(1, std::memory_order_relaxed);
     }
     return cudaPeekAtLastError() == cudaSuccess ? FLORA_OK : FLORA_ERR_CUDA;
@@ -941,7 +931,7 @@ inline flora_status tc_decompress_single(flora_mat* W, const flora_mat* S, uint6
 
 inline bool tc_decompress_supported(const flora_mat* big, const flora_mat* sketch)
 {
-    return tc_mat_ok(*big) && sketch->cols >= 1 && sketch->cols <= 256 && encode_tiled_fn() != nullptr;
+    return tc_mat_ok(*big) && tc_sketch_ok(*sketch) && encode_tiled_fn() != nullptr;
 }
 
 inline flora_status tc_set_zero(TcSet& set, cudaStream_t st, std::atomic<uint64_t>& launches)
