@@ -95,6 +95,28 @@ flora_status flora_momentum_step(const flora_mat* G, flora_mat* M, float beta, u
  * returned to it before the call returns; FLORA_ERR_ALLOC if that fails. */
 flora_status flora_resample_transfer(flora_mat* M, int64_t m, int32_t operand, uint64_t seed_old, uint64_t seed_new, void* stream);
 
+/* The same operation as flora_resample_transfer for callers that must not allocate.  (The paper has no
+ * counterpart to this call: it is a packaging of Algorithm 2's transfer for a constrained caller.)
+ *
+ * flora_resample_transfer borrows its r x r scratch from cudaMallocAsync.  That is unusable for code that
+ * runs after all device memory has been handed out (an inference or training process whose memory plan is
+ * fixed up front and which treats any later allocation as a failure), for code that may not touch the
+ * allocator at all at this point (a latency-critical loop, a thread that does not own the memory pool), and
+ * wherever an allocation call could block or fail at an inconvenient time.  This variant calls neither
+ * cudaMalloc / cudaFree nor their stream-ordered forms, nor any library routine that allocates: its scratch
+ * is a fixed array of 256 x 256 floats (256 KB) inside the library image, so every GPU on which the library
+ * is used holds those 256 KB until the process exits, whether or not this call is ever made.
+ *
+ *  - Limit: r = M->cols <= 256 (the scratch size); a larger r returns FLORA_ERR_RANK and launches nothing.
+ *  - The first call on each device looks up the device address of the array (cudaGetSymbolAddress, with
+ *    that device current); make that first call outside any stream capture.  Later calls only launch.
+ *  - All calls on a device share the one array, and it keeps what the last call left in it.  The call clears
+ *    it first (a memset on `stream`), so back-to-back calls on one stream are fine; two calls that may run
+ *    concurrently on the same GPU (different streams, different threads) race on the array and must be
+ *    serialised by the caller.
+ * Arguments, result and error codes are otherwise those of flora_resample_transfer. */
+flora_status flora_resample_transfer_static(flora_mat* M, int64_t m, int32_t operand, uint64_t seed_old, uint64_t seed_new, void* stream);
+
 /* dst <- b dst + a src A(seed_old) A(seed_new)^T.  With a = (1-beta)/tau, b = beta this feeds the
  * output of Algorithm 1 (G~ = C A_acc / tau) into the update of Algorithm 2 without forming G~.
  * dst, src: n x r f32; they may be the same matrix.  Scratch as for flora_resample_transfer. */

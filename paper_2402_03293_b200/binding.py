@@ -25,7 +25,7 @@ FLORA_F32, FLORA_BF16 = 0, 1
 # every symbol include/flora.h declares
 EXPORTS = [
     "flora_compress_accumulate", "flora_decompress_apply", "flora_momentum_step", "flora_resample_transfer",
-    "flora_transfer_axpby", "flora_materialize_A", "flora_set_create", "flora_set_destroy",
+    "flora_resample_transfer_static", "flora_transfer_axpby", "flora_materialize_A", "flora_set_create", "flora_set_destroy",
     "flora_set_rebind_gradients", "flora_set_compress_accumulate", "flora_set_momentum_step",
     "flora_set_decompress_apply", "flora_set_resample_transfer", "flora_set_zero_state", "flora_derive_seed",
     "flora_resamples_at", "flora_set_compress_accumulate_from_host", "flora_set_read_weights_to_host",
@@ -61,6 +61,7 @@ def load() -> ctypes.CDLL:
             "flora_decompress_apply": (I32, [MP, MP, U64, F, F, P]),
             "flora_momentum_step": (I32, [MP, MP, F, U64, P]),
             "flora_resample_transfer": (I32, [MP, I64, I32, U64, U64, P]),
+            "flora_resample_transfer_static": (I32, [MP, I64, I32, U64, U64, P]),
             "flora_transfer_axpby": (I32, [MP, MP, I64, I32, U64, U64, F, F, P]),
             "flora_materialize_A": (I32, [MP, U64, P]),
             "flora_set_create": (I32, [ctypes.c_int, MP, MP, MP, ctypes.POINTER(P)]),
@@ -155,6 +156,14 @@ def flora_resample_transfer(M: torch.Tensor, m: int, operand, seed_old: int, see
     m_ = mat(M)
     _check(load().flora_resample_transfer(ctypes.byref(m_), m, _dt(operand), seed_old, seed_new, _stream(stream)),
            "flora_resample_transfer")
+
+
+def flora_resample_transfer_static(M: torch.Tensor, m: int, operand, seed_old: int, seed_new: int, stream=None) -> None:
+    """flora_resample_transfer without any allocation: the r x r scratch is a fixed 256 KB array inside the
+    library (r <= 256).  Calls that can overlap on one GPU must be serialised by the caller."""
+    m_ = mat(M)
+    _check(load().flora_resample_transfer_static(ctypes.byref(m_), m, _dt(operand), seed_old, seed_new, _stream(stream)),
+           "flora_resample_transfer_static")
 
 
 def flora_transfer_axpby(dst: torch.Tensor, src: torch.Tensor, m: int, operand, seed_old: int, seed_new: int,

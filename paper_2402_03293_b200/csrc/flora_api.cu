@@ -8,6 +8,7 @@
 #include <string.h>
 
 #include <atomic>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -140,6 +141,35 @@ flora_status transfer_with_scratch(flora_mat* dst, const flora_mat* src, int64_t
     return simt_apply_gram(dst, src, T, a, b, st);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Scratch for flora_resample_transfer_static: lives in the library image, one copy per GPU that loads it.
+// In host code the name below is only a handle; the device address comes from cudaGetSymbolAddress.
+// ------------------------------------------------------------------------------------------------
+constexpr int STATIC_TRANSFER_MAX_R = 256;
+static __device__ __align__(256) float g_static_transfer_scratch[STATIC_TRANSFER_MAX_R * STATIC_TRANSFER_MAX_R];
+
+constexpr int MAX_DEVICES = 64;
+std::mutex g_static_mutex;
+float* g_static_scratch_addr[MAX_DEVICES] = {};
+
+// Device address of the scratch on the current device, looked up once per device.
+flora_status static_scratch_for_current_device(float** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return FLORA_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_scratch_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_transfer_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return FLORA_ERR_CUDA;
+        }
+        g_static_scratch_addr[dev] = static_cast<float*>(p);
+    }
+    *out = g_static_scratch_addr[dev];
+    return FLORA_OK;
+}
+
 bool use_tc_compress(const flora_mat* big, const flora_mat* sketch)
 {
     return g_force_path.load(std::memory_order_relaxed) != 1 && tc_compress_supported(big, sketch);
@@ -211,6 +241,20 @@ flora_status flora_transfer_axpby(flora_mat* dst, const flora_mat* src, int64_t 
 flora_status flora_resample_transfer(flora_mat* M, int64_t m, int32_t operand, uint64_t seed_old, uint64_t seed_new, void* stream)
 {
     return flora_transfer_axpby(M, M, m, operand, seed_old, seed_new, 1.0f, 0.0f, stream);
+}
+
+flora_status flora_resample_transfer_static(flora_mat* M, int64_t m, int32_t operand, uint64_t seed_old, uint64_t seed_new, void* stream)
+{
+    flora_status st = check_transfer(M, M, m, operand);
+    if (st) return st;
+    const int64_t r = M->cols;
+    if (r * r > (int64_t)STATIC_TRANSFER_MAX_R * STATIC_TRANSFER_MAX_R) return FLORA_ERR_RANK;   // larger than the built-in scratch
+    if (M->rows == 0) return FLORA_OK;
+    float* T = nullptr;
+    st = static_scratch_for_current_device(&T);
+    if (st) return st;
+    // T is cleared inside (it still holds the previous call's product), then filled and applied
+    return transfer_with_scratch(M, M, m, operand, seed_old, seed_new, 1.0f, 0.0f, T, as_stream(stream));
 }
 
 flora_status flora_materialize_A(flora_mat* out, uint64_t seed, void* stream)
