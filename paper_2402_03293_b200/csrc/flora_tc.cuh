@@ -64,12 +64,14 @@ struct SeedTable {
 // r x 64 tile of A (bf16) into shared memory; one thread issues tiles x 4 MMAs (128 x r_pad x 16)
 // that accumulate in tensor memory.  At the end four warps read the accumulators back and update S.
 // ------------------------------------------------------------------------------------------------
-constexpr int K1_GEN_WARPS = 8;
-constexpr int K1_THREADS = 64 + 32 * K1_GEN_WARPS;
+constexpr int K1_MAX_GEN_WARPS = 16;
+constexpr int K1_MAX_THREADS = 64 + 32 * K1_MAX_GEN_WARPS + 32;
+// threads of a CTA: producer warp, MMA warp, GW generator warps, one warp that forwards slices to cluster peers
+inline int k1_threads(int gen_warps) { return 64 + 32 * gen_warps + 32; }
 constexpr int G_TILE_BYTES = 128 * 128;   // 128 rows x 64 bf16
 
 struct K1Smem {                            // barriers and scalars, placed after the tile ring
-    uint64_t full_g[8], full_a[8], empty[8], acc_full;
+    uint64_t full_g[8], full_a[8], slice_ready[8], empty[8], acc_full;
     uint32_t tmem_base;
     int abort;
 };
@@ -107,9 +109,9 @@ __device__ __forceinline__ void k1_store_chunk(float* srow, const uint32_t (&v)[
     }
 }
 
-__global__ void __launch_bounds__(K1_THREADS, 1)
+__global__ void __launch_bounds__(K1_MAX_THREADS, 1)
 compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__ items, const __grid_constant__ SeedTable seeds,
-                   int seed_base, int r, float scale, float a, float b, int T, int stages)
+                   int seed_base, int r, float scale, float a, float b, int T, int stages, int S, int GW)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
@@ -127,8 +129,9 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->full_g[s]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctl->full_a[s]), K1_GEN_WARPS);
-            ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctl->full_a[s]), S > 1 ? 1 : GW);   // cluster: one arrival + the peers' bytes
+            ptx::mbar_init(ptx::smem_addr(&ctl->slice_ready[s]), GW);
+            ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), S);                   // every CTA of the cluster has consumed the stage
         }
         ptx::mbar_init(ptx::smem_addr(&ctl->acc_full), 1);
         ctl->abort = 0;
@@ -143,24 +146,28 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
     if (r_pad > r) {
         const int pad_chunks = (r_pad - r) * 8;
         for (int s = 0; s < stages; ++s)
-            for (int t = threadIdx.x; t < pad_chunks; t += K1_THREADS)
+            for (int t = threadIdx.x; t < pad_chunks; t += (int)blockDim.x)
                 ptx::st_shared_v4(smem_base + s * stage_bytes + T * G_TILE_BYTES + (uint32_t)r * 128u + t * 16u, 0, 0, 0, 0);
         ptx::fence_proxy_async_smem();
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (S > 1) ptx::cluster_sync();       // every CTA's barriers exist before anyone arrives on them remotely
     ptx::tc_fence_after_sync();
     const uint32_t tmem = ctl->tmem_base;
     volatile int* abort = &ctl->abort;
+    const uint32_t rank = S > 1 ? ptx::cluster_ctarank() : 0u;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        if (lane == 0 && item.tiles > 0) {
             ptx::prefetch_tensormap(&mat->map_g);
             int issued = 0;
             for (int ks = 0; ks < item.ksteps; ++ks) {
                 const int s = ks % stages, it = ks / stages;
-                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort)) break;
+                if (!(S > 1 ? ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort)
+                            : ptx::mbar_wait(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort)))
+                    break;
                 const uint32_t bar = ptx::smem_addr(&ctl->full_g[s]);
                 ptx::mbar_arrive_expect_tx(bar, (uint32_t)item.tiles * G_TILE_BYTES);
                 for (int t = 0; t < item.tiles; ++t)
@@ -181,8 +188,9 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
             bool ok = true;
             for (int ks = 0; ks < item.ksteps && ok; ++ks) {
                 const int s = ks % stages, it = ks / stages;
-                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[s]), it & 1, abort) &&
-                     ptx::mbar_wait(ptx::smem_addr(&ctl->full_a[s]), it & 1, abort);
+                ok = (item.tiles == 0 || ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[s]), it & 1, abort)) &&
+                     (S > 1 ? ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->full_a[s]), it & 1, abort)
+                            : ptx::mbar_wait(ptx::smem_addr(&ctl->full_a[s]), it & 1, abort));
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t stage = smem_base + s * stage_bytes;
@@ -194,33 +202,71 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
                                        ptx::umma_desc_k_sw128(a_tile + kk * 32), idesc, (ks | kk) != 0);
                     }
                 }
-                ptx::umma_commit(ptx::smem_addr(&ctl->empty[s]));
+                // the stage is free once every CTA of the cluster has consumed its copy of the A tile
+                const uint32_t ebar = ptx::smem_addr(&ctl->empty[s]);
+                if (S == 1) ptx::umma_commit(ebar);
+                else if (item.tiles > 0) ptx::umma_commit_cluster(ebar, (uint16_t)((1u << S) - 1u));
+                else
+                    for (int d = 0; d < S; ++d) ptx::mbar_arrive_cluster(ptx::map_to_cta(ebar, d));   // a CTA without rows consumes nothing
             }
-            if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->acc_full));
+            if (ok && item.tiles > 0) ptx::umma_commit(ptx::smem_addr(&ctl->acc_full));
+        }
+    } else if (warp == 2 + GW) {
+        // ------------------------------------------------------------------ forwarder: this CTA's slice of A to the peers
+        if (lane == 0 && S > 1) {
+            const uint32_t slice_bytes = (uint32_t)(r_pad / S) * 128u;
+            for (int ks = 0; ks < item.ksteps; ++ks) {
+                const int s = ks % stages, it = ks / stages;
+                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->slice_ready[s]), it & 1, abort)) break;
+                const uint32_t fbar = ptx::smem_addr(&ctl->full_a[s]);
+                const uint32_t src = smem_base + s * stage_bytes + T * G_TILE_BYTES + rank * slice_bytes;
+                ptx::mbar_arrive_expect_tx(fbar, (uint32_t)(S - 1) * slice_bytes);   // own slice is in place; peers' bytes to come
+                for (int d = 0; d < S; ++d)
+                    if (d != (int)rank) ptx::bulk_copy_to_peer(ptx::map_to_cta(src, d), src, slice_bytes, ptx::map_to_cta(fbar, d));
+            }
         }
     } else {
         // ------------------------------------------------------------------ generators, then epilogue
-        const int g = threadIdx.x - 64;                       // 0 .. 32*K1_GEN_WARPS-1
+        const int g = threadIdx.x - 64;                       // 0 .. 32*GW-1
         const PhiloxKey key = make_key(seeds.s[item.mat - seed_base]);
         const int tasks = r * 8;                              // (row j, 16-byte chunk c) pairs of one A tile
         bool ok = true;
         for (int ks = 0; ks < item.ksteps && ok; ++ks) {
             const int s = ks % stages, it = ks / stages;
-            ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort);
+            ok = S > 1 ? ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort)
+                       : ptx::mbar_wait(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort);
             if (!ok) break;
             const uint32_t a_tile = smem_base + s * stage_bytes + T * G_TILE_BYTES;
             const uint32_t q0 = (uint32_t)(item.kstep0 + ks) * 16u;
-            for (int t = g; t < tasks; t += 32 * K1_GEN_WARPS) {
-                const int j = t >> 3, c = t & 7;
-                const uint2 lo = projection_quad_bf16(q0 + 2 * c, (uint32_t)j, key, scale);
-                const uint2 hi = projection_quad_bf16(q0 + 2 * c + 1, (uint32_t)j, key, scale);
-                ptx::st_shared_v4(a_tile + j * 128 + ((c ^ (j & 7)) << 4), lo.x, lo.y, hi.x, hi.y);
+            if (S == 1) {
+                for (int t = g; t < tasks; t += 32 * GW) {
+                    const int j = t >> 3, c = t & 7;
+                    const uint2 lo = projection_quad_bf16(q0 + 2 * c, (uint32_t)j, key, scale);
+                    const uint2 hi = projection_quad_bf16(q0 + 2 * c + 1, (uint32_t)j, key, scale);
+                    ptx::st_shared_v4(a_tile + j * 128 + ((c ^ (j & 7)) << 4), lo.x, lo.y, hi.x, hi.y);
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->full_a[s]));
+            } else {
+                // the CTAs of a cluster work on the same columns of the same matrix: each generates the rows
+                // [rank, rank+1) * r_pad/S of the tile in its own shared memory; the forwarder warp sends them on
+                const int rows_per_cta = r_pad / S;
+                const int my_tasks = rows_per_cta * 8;
+                for (int t = g; t < my_tasks; t += 32 * GW) {
+                    const int j = (int)rank * rows_per_cta + (t >> 3), c = t & 7;
+                    if (j < r) {
+                        const uint2 lo = projection_quad_bf16(q0 + 2 * c, (uint32_t)j, key, scale);
+                        const uint2 hi = projection_quad_bf16(q0 + 2 * c + 1, (uint32_t)j, key, scale);
+                        ptx::st_shared_v4(a_tile + j * 128 + ((c ^ (j & 7)) << 4), lo.x, lo.y, hi.x, hi.y);
+                    }
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->slice_ready[s]));
             }
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->full_a[s]));
         }
-        if (warp < 6 && ok) {
+        if (warp < 6 && ok && item.tiles > 0) {
             // epilogue: warp w reads tensor-memory lanes 32*(w%4) .. +31, i.e. rows of the tile
             const int quarter = warp & 3;
             if (ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full), 0, abort)) {
@@ -249,6 +295,7 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (S > 1) ptx::cluster_sync();       // no CTA leaves while peers may still store into it or arrive on its barriers
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem, tmem_cols);
@@ -517,7 +564,8 @@ struct TcSet {
     bool decompress_ready = false;
     bool transient = false;             // device buffers come from the stream-ordered allocator
     int count = 0, r = 0;
-    int T = 1, stages = 2;
+    int T = 1, stages = 2, S = 1, GW = 8;
+    std::vector<int> k1_launch_first_mat;
     size_t k1_smem = 0;
     TcMatrix* d_mats = nullptr;
     K1Item* d_k1 = nullptr;
@@ -621,6 +669,11 @@ inline int tune_knob(const char* name, int dflt, int lo, int hi)
 }
 
 // Work decomposition of the compression kernel over a set of matrices.
+//
+// A CTA handles up to T 128-row tiles; S CTAs (a thread-block cluster) handle neighbouring row groups of the
+// same matrix over the same columns and share the generation of A.  The generation of one r x 64 tile costs
+// about r*64*0.18 ns of one SM's ALUs, the loads of a CTA's T tiles T*0.37 us of its share of HBM: S is chosen
+// so that the former stays under half of the latter.
 inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
 {
     const int r_pad = (r + 15) & ~15;
@@ -630,71 +683,161 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
         max_tiles = std::max(max_tiles, tiles);
         total_work += tiles * ks;
     }
-    // T: row tiles per CTA.  More tiles amortise the generation of A (one r x 64 tile serves T x 128 rows);
-    // bounded by tensor memory (T * r_pad <= 512 columns) and by shared memory.  Among the allowed values
-    // take the one that wastes the fewest tile slots over the set, the larger one on a tie.
-    const int t_cap = (int)std::min<int64_t>(std::min<int64_t>(max_tiles, 512 / r_pad), 4);
-    int T = 1;
-    double best = 1e300;
-    for (int cand = t_cap; cand >= 1; --cand) {
+    // T: bounded by tensor memory (T * r_pad <= 512 columns).  The largest value, unless a smaller one removes
+    // more than a fifth of the tile slots that row counts which are no multiple of T * 128 leave empty
+    // (empty slots cost MMA issue and shared memory, not HBM traffic).
+    // (for r <= 32 at most 3 tiles, so that two CTAs with two stages each fit one SM)
+    const int t_cap = (int)std::min<int64_t>(std::min<int64_t>(max_tiles, 512 / r_pad), r_pad <= 32 ? 3 : 4);
+    auto padded_work = [&](int cand) {
         double padded = 0;
         for (const auto& g : G) {
             const int64_t tiles = (g.rows + 127) / 128, ks = (g.cols + 63) / 64;
             padded += (double)((tiles + cand - 1) / cand * cand) * ks;
         }
-        if (padded < best * 0.999) {
-            best = padded;
-            T = cand;
-        }
-    }
+        return padded;
+    };
+    int T = t_cap;
+    for (int cand = t_cap - 1; cand >= 1; --cand)
+        if (padded_work(cand) < 0.8 * padded_work(T)) T = cand;
     T = tune_knob("FLORA_K1_T", T, 1, 512 / r_pad);
     const size_t stage = (size_t)T * G_TILE_BYTES + (size_t)r_pad * 128;
     uint32_t cols = 32;
     while ((int)cols < T * r_pad) cols <<= 1;
+    // cluster size from the generation / load ratio
+    const double ratio = r * 0.0305 / T;
+    int S = 1;
+    while (S < 8 && ratio / S > 0.5) S <<= 1;
+    while (S > 1 && (int64_t)S * T > 2 * max_tiles) S >>= 1;         // not more CTAs than there are rows to share
+    S = tune_knob("FLORA_K1_CLUSTER", S, 1, 8);
+    if (S & (S - 1)) S = 1;
+    while (S > 1 && r_pad % (8 * S)) S >>= 1;                     // every CTA's slice of A is whole 8-row groups
     // two CTAs per SM when tensor memory allows it and each still gets two stages: the epilogue of one
-    // overlaps the loads of the other
-    int per_sm = (cols <= 256 && 2 * stage <= SMEM_BUDGET / 2) ? 2 : 1;
-    per_sm = tune_knob("FLORA_K1_PER_SM", per_sm, 1, cols <= 256 ? 2 : 1);
+    // overlaps the loads of the other (single-CTA clusters only)
+    int per_sm = (S == 1 && cols <= 256 && 2 * stage <= SMEM_BUDGET / 2) ? 2 : 1;
+    per_sm = tune_knob("FLORA_K1_PER_SM", per_sm, 1, (S == 1 && cols <= 256) ? 2 : 1);
     int stages = (int)std::min<size_t>(8, SMEM_BUDGET / per_sm / stage);
     stages = tune_knob("FLORA_K1_STAGES", stages, 1, std::max(1, stages));
+    // generator warps: 16 where one CTA owns the SM and generation is a sizeable share of the work
+    int GW = (per_sm == 1 && ratio / S > 0.15) ? 16 : 8;
+    GW = tune_knob("FLORA_K1_GEN_WARPS", GW, 4, per_sm == 1 ? K1_MAX_GEN_WARPS : 8);
+    set.GW = GW;
     set.T = T;
+    set.S = S;
     set.stages = stages;
     set.k1_smem = (size_t)stages * stage + sizeof(K1Smem) + 1024;
-    // column chunks: aim at about `waves` items per CTA slot, at least 8 steps (512 columns) per item
-    const int64_t slots = (int64_t)sm_count() * per_sm;
-    const int waves = tune_knob("FLORA_K1_WAVES", 1, 1, 64);
-    const int64_t target = std::max<int64_t>(8 * T, total_work / (waves * slots) + 1);
-    set.h_k1.clear();
-    set.split_mats.clear();
-    for (size_t i = 0; i < G.size(); ++i) {
-        const auto& g = G[i];
-        if (g.rows == 0 || g.cols == 0) continue;
-        const int64_t tiles = (g.rows + 127) / 128, ks = (g.cols + 63) / 64;
-        int64_t chunk = std::max<int64_t>(8, target / T);
-        int64_t nchunks = (ks + chunk - 1) / chunk;
-        if (nchunks > 1 && ks - (nchunks - 1) * chunk < chunk / 2) --nchunks;    // no short tail item
-        chunk = (ks + nchunks - 1) / nchunks;
-        nchunks = (ks + chunk - 1) / chunk;
-        if (nchunks > 1) set.split_mats.push_back((int)i);
-        for (int64_t t0 = 0; t0 < tiles; t0 += T)
-            for (int64_t c = 0; c < nchunks; ++c) {
-                K1Item it;
-                it.mat = (int)i;
-                it.row0 = (int)(t0 * 128);
-                it.tiles = (int)std::min<int64_t>(T, tiles - t0);
-                it.kstep0 = (int)(c * chunk);
-                it.ksteps = (int)std::min<int64_t>(chunk, ks - c * chunk);
-                it.direct = nchunks == 1;
-                set.h_k1.push_back(it);
-            }
+    // column chunks: aim at about `waves` items per slot (a slot is a CTA, or a cluster), at least 8 steps each
+    int64_t slots = std::max<int64_t>(1, (int64_t)sm_count() * per_sm / S);
+    cudaFuncSetAttribute(compress_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)set.k1_smem);
+    if (S > 1) {
+        // clusters that can be resident at once (fewer than SMs / S: a cluster must sit inside one GPC)
+        cudaFuncSetAttribute(compress_tc_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 0);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(S * 64));
+        cfg.blockDim = dim3((unsigned)k1_threads(set.GW));
+        cfg.dynamicSmemBytes = set.k1_smem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)S;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int active = 0;
+        if (cudaOccupancyMaxActiveClusters(&active, compress_tc_kernel, &cfg) == cudaSuccess && active > 0) slots = active;
+        else cudaGetLastError();
     }
-    set.k1_launch_begin.clear();
-    int begin_mat = -1;
-    for (size_t k = 0; k < set.h_k1.size(); ++k) {
-        if (begin_mat < 0 || set.h_k1[k].mat >= begin_mat + SEEDS_PER_LAUNCH) {
-            begin_mat = set.h_k1[k].mat;
-            set.k1_launch_begin.push_back((int)k);
+    const int64_t group_tiles = (int64_t)S * T;                      // rows of one slot, in tiles
+    struct Unit { int mat; int64_t tile0, tiles, kstep0, ksteps; bool direct; };
+    auto build_units = [&](int64_t target, std::vector<Unit>& units, std::vector<int>& split) {
+        units.clear();
+        split.clear();
+        for (size_t i = 0; i < G.size(); ++i) {
+            const auto& g = G[i];
+            if (g.rows == 0 || g.cols == 0) continue;
+            const int64_t tiles = (g.rows + 127) / 128, ks = (g.cols + 63) / 64;
+            const int64_t groups = (tiles + group_tiles - 1) / group_tiles;
+            const int64_t per_group = (tiles + groups - 1) / groups;     // rows spread evenly over the groups
+            int64_t chunk = std::max<int64_t>(8, target / per_group);
+            int64_t nchunks = (ks + chunk - 1) / chunk;
+            if (nchunks > 1 && ks - (nchunks - 1) * chunk < chunk / 2) --nchunks;    // no short tail item
+            chunk = (ks + nchunks - 1) / nchunks;
+            nchunks = (ks + chunk - 1) / chunk;
+            if (nchunks > 1) split.push_back((int)i);
+            for (int64_t t0 = 0; t0 < tiles; t0 += per_group)
+                for (int64_t c = 0; c < nchunks; ++c)
+                    units.push_back({(int)i, t0, std::min(per_group, tiles - t0), c * chunk, std::min(chunk, ks - c * chunk), nchunks == 1});
         }
+    };
+    // time of a unit on its slot, in 64-column steps of a full slot: a fixed start-up / epilogue cost plus its steps,
+    // scaled by the rows a CTA streams (a cluster moves in lockstep, so its most loaded CTA counts)
+    auto unit_time = [&](const Unit& u) {
+        const double per_cta = (double)((u.tiles + S - 1) / S);
+        return (6.0 + (double)u.ksteps) * std::max(per_cta, 0.5 * T);
+    };
+    auto makespan = [&](const std::vector<Unit>& units) {
+        std::vector<double> tms;
+        for (const auto& u : units) tms.push_back(unit_time(u));
+        std::sort(tms.begin(), tms.end(), std::greater<double>());
+        std::vector<double> free_at((size_t)slots, 0.0);     // min-heap of slot availability
+        auto cmp = std::greater<double>();
+        for (double t : tms) {
+            std::pop_heap(free_at.begin(), free_at.end(), cmp);
+            free_at.back() += t;
+            std::push_heap(free_at.begin(), free_at.end(), cmp);
+        }
+        return *std::max_element(free_at.begin(), free_at.end());
+    };
+    // column chunks: try several granularities (about 1..4 units per slot) and keep the shortest schedule
+    std::vector<Unit> units, cand_units;
+    std::vector<int> cand_split;
+    double best_span = 1e300;
+    const int fixed_waves = tune_knob("FLORA_K1_WAVES", 0, 0, 64);
+    for (int w = 1; w <= 4; ++w) {
+        for (double f : {1.0, 1.1, 1.2, 1.35, 1.5}) {
+            if (fixed_waves && (w != fixed_waves || f != 1.0)) continue;
+            const int64_t target = (int64_t)((double)total_work / (double)((fixed_waves ? fixed_waves : w) * slots) * f) + 1;
+            build_units(target, cand_units, cand_split);
+            const double span = makespan(cand_units);
+            if (span < best_span * 0.98) {
+                best_span = span;
+                units = cand_units;
+                set.split_mats = cand_split;
+            }
+        }
+    }
+    // launches cover at most SEEDS_PER_LAUNCH consecutive matrices; inside a launch the largest units go first
+    set.h_k1.clear();
+    set.k1_launch_begin.clear();
+    set.k1_launch_first_mat.clear();
+    size_t u0 = 0;
+    while (u0 < units.size()) {
+        size_t u1 = u0;
+        while (u1 < units.size() && units[u1].mat < units[u0].mat + SEEDS_PER_LAUNCH) ++u1;
+        const int first_mat = units[u0].mat;          // before sorting: units are still in matrix order here
+        if (tune_knob("FLORA_K1_SORT", 1, 0, 1))
+            std::stable_sort(units.begin() + u0, units.begin() + u1,
+                             [](const Unit& x, const Unit& y) { return x.tiles * x.ksteps > y.tiles * y.ksteps; });
+        set.k1_launch_begin.push_back((int)set.h_k1.size());
+        set.k1_launch_first_mat.push_back(first_mat);
+        for (size_t u = u0; u < u1; ++u) {
+            // the unit's tiles spread evenly over the S CTAs of the slot (some may get none)
+            const Unit& un = units[u];
+            int64_t t0 = un.tile0;
+            for (int c = 0; c < S; ++c) {
+                const int64_t left = un.tile0 + un.tiles - t0;
+                const int64_t mine = std::min<int64_t>(T, (left + (S - c) - 1) / (S - c));
+                K1Item it;
+                it.mat = un.mat;
+                it.row0 = (int)(t0 * 128);
+                it.tiles = (int)std::max<int64_t>(0, mine);
+                it.kstep0 = (int)un.kstep0;
+                it.ksteps = (int)un.ksteps;
+                it.direct = un.direct;
+                set.h_k1.push_back(it);
+                t0 += it.tiles;
+            }
+        }
+        u0 = u1;
     }
     set.k1_launch_begin.push_back((int)set.h_k1.size());
 }
@@ -879,11 +1022,26 @@ inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, 
     for (size_t l = 0; l + 1 < set.k1_launch_begin.size(); ++l) {
         const int begin = set.k1_launch_begin[l], end = set.k1_launch_begin[l + 1];
         if (end == begin) continue;
-        const int seed_base = set.h_k1[begin].mat;
+        const int seed_base = set.k1_launch_first_mat[l];
         SeedTable table;
         for (int i = 0; i < SEEDS_PER_LAUNCH; ++i) table.s[i] = seed_base + i < set.count ? seeds[seed_base + i] : 0;
-        compress_tc_kernel<<<end - begin, K1_THREADS, set.k1_smem, st>>>(set.d_mats, set.d_k1 + begin, table, seed_base, r, scale,
-                                                                         a, b, set.T, set.stages);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(end - begin));
+        cfg.blockDim = dim3((unsigned)k1_threads(set.GW));
+        cfg.dynamicSmemBytes = set.k1_smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)set.S;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = set.S > 1 ? 1 : 0;
+        const TcMatrix* mats = set.d_mats;
+        const K1Item* items = set.d_k1 + begin;
+        if (cudaLaunchKernelEx(&cfg, compress_tc_kernel, mats, items, table, seed_base, r, scale, a, b, set.T, set.stages, set.S, set.GW) !=
+            cudaSuccess)
+            return FLORA_ERR_CUDA;
         launches.fetch_add(1, std::memory_order_relaxed);
     }
     return cudaPeekAtLastError() == cudaSuccess ? FLORA_OK : FLORA_ERR_CUDA;

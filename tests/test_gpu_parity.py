@@ -47,7 +47,7 @@ def test_generated_projection_is_bit_exact(seed, r, m):
 SHAPES = [(1, 1, 1), (5, 7, 3), (33, 100, 8), (130, 257, 17), (64, 512, 32), (300, 1000, 64), (129, 200, 256),
           # eligible for the tensor-core kernels (bf16, 16-byte aligned rows, n >= 128, m >= 64), ragged tiles and tails
           (128, 64, 16), (256, 1024, 32), (1000, 2056, 8), (384, 4104, 32), (515, 1288, 128), (200, 776, 96),
-          (700, 1600, 256), (1030, 520, 1)]
+          (700, 1600, 256), (1030, 520, 1), (2100, 1088, 256), (1600, 1600, 200)]
 
 
 @pytest.mark.parametrize("force_simt", [0, 1])
