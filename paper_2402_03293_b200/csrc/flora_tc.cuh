@@ -305,14 +305,18 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
 // ------------------------------------------------------------------------------------------------
 // decompression fused with the update:  W <- W - step * S A
 //
-// One CTA owns a slab of `bn` (128 or 64) columns of one matrix and `tiles` 128-row tiles of it.
-// It generates the r x bn slab of A once (the N x K operand: bf16 values held in 32-bit containers)
-// and then streams row tiles: TMA brings the fp32 rows of S in 32-column chunks and the W tile into
-// shared memory; one thread issues tf32 MMAs (128 x bn x 8) that read S as it is stored, into one of
-// two tensor-memory accumulators; four warps combine the accumulator with the W tile in shared memory
-// and a TMA store writes the tile back.  W is read once and written once, S is never converted.
+// Persistent kernel: CTA c processes the work items c, c + gridDim.x, ...  An item is a slab of `bn` (128 or 64)
+// columns of one matrix and a run of 128-row tiles.  Per item the generator warps write the r x bn slab of A
+// (the N x K operand: bf16 values held in 32-bit containers) into one of two slab buffers, so the slab of the
+// next item is generated while the current one streams.  Per row tile: TMA brings the fp32 rows of S in
+// 32-column chunks and the W tile into shared memory; one thread issues tf32 MMAs (128 x bn x 8) that read S
+// as it is stored, into one of two tensor-memory accumulators; four warps combine the accumulator with the W
+// tile in shared memory and a TMA store writes the tile back.  W is read once and written once.
+// All rings (W slots, S chunks, accumulators, slabs) run across item boundaries.
 // ------------------------------------------------------------------------------------------------
-constexpr int K2_THREADS = 256;   // warp 0: W loads, 1: MMA, 2-5: combine, 6: S loads, 7: W stores
+constexpr int K2_FIXED_WARPS = 8;   // warp 0: W loads, 1: MMA, 2-5: combine, 6: S loads, 7: W stores, 8..: slab generators
+constexpr int K2_MAX_GEN_WARPS = 8;
+constexpr int K2_MAX_THREADS = 32 * (K2_FIXED_WARPS + K2_MAX_GEN_WARPS);
 constexpr int K2_MAX_SLOTS = 6;
 constexpr int K2_MAX_CSTAGES = 8;
 constexpr int W_BOX_BYTES = 128 * 128;     // 128 rows x 64 bf16
@@ -320,31 +324,29 @@ constexpr int S_CHUNK_BYTES = 128 * 128;   // 128 rows x 32 fp32
 
 struct K2Smem {
     uint64_t w_full[K2_MAX_SLOTS], w_free[K2_MAX_SLOTS], out_ready[K2_MAX_SLOTS];
-    uint64_t c_full[K2_MAX_CSTAGES], c_empty[K2_MAX_CSTAGES], acc_full[2], acc_empty[2];
+    uint64_t c_full[K2_MAX_CSTAGES], c_empty[K2_MAX_CSTAGES], acc_full[2], acc_empty[2], slab_full[2], slab_empty[2];
     uint32_t tmem_base;
     int abort;
 };
 
-__global__ void __launch_bounds__(K2_THREADS, 1)
-decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict__ items, const __grid_constant__ SeedTable seeds,
-                     int seed_base, int r, float scale, float step, int bn, int slots, int cstages)
+__global__ void __launch_bounds__(K2_MAX_THREADS, 1)
+decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict__ items, int n_items,
+                     const __grid_constant__ SeedTable seeds, int seed_base, int r, float scale, float step, int bn, int slots,
+                     int cstages, int GW)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
     const int kchunks = (r + 31) >> 5;                         // 32-deep K chunks (one 128-byte row of fp32 each)
     const int boxes = bn >> 6;                                 // 64-column boxes per W tile
-    const uint32_t slab_block = (uint32_t)bn * 128u;           // one K chunk of the slab
-    const uint32_t slab = smem_base;
-    const uint32_t c_ring = slab + kchunks * slab_block;
+    const uint32_t slab_block = (uint32_t)bn * 128u;           // one K chunk of a slab
+    const uint32_t slab_bytes = kchunks * slab_block;
+    const uint32_t slab0 = smem_base;
+    const uint32_t c_ring = slab0 + 2 * slab_bytes;
     const uint32_t w_ring = c_ring + cstages * (uint32_t)S_CHUNK_BYTES;
     const uint32_t slot_bytes = (uint32_t)boxes * W_BOX_BYTES;
     K2Smem* ctl = reinterpret_cast<K2Smem*>(smem_raw + (w_ring - ptx::smem_addr(smem_raw)) + (size_t)slots * slot_bytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-    const K2Item item = items[blockIdx.x];
-    const TcMatrix* mat = mats + item.mat;
     const uint32_t tmem_cols = 2u * (uint32_t)bn;              // 256 or 128: a power of two >= 32
-    const int live_boxes = min(boxes, (mat->m - item.col0 + 63) >> 6);   // boxes that overlap the matrix
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < slots; ++s) {
@@ -359,6 +361,8 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->acc_full[s]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[s]), 4);
+            ptx::mbar_init(ptx::smem_addr(&ctl->slab_full[s]), GW);
+            ptx::mbar_init(ptx::smem_addr(&ctl->slab_empty[s]), 1);
         }
         ctl->abort = 0;
         ptx::fence_barrier_init();
@@ -374,158 +378,183 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
     const uint32_t tmem = ctl->tmem_base;
     volatile int* abort = &ctl->abort;
 
-    // The first W tiles and S chunks are requested before the slab is generated (fresh slots: nothing to wait for).
-    const int total_chunks = item.tiles * kchunks;
-    auto load_w = [&](int i) {
-        const int s = i % slots;
-        const uint32_t bar = ptx::smem_addr(&ctl->w_full[s]);
-        ptx::mbar_arrive_expect_tx(bar, (uint32_t)live_boxes * W_BOX_BYTES);
-        for (int bx = 0; bx < live_boxes; ++bx)
-            ptx::tma_load_2d(w_ring + s * slot_bytes + bx * W_BOX_BYTES, &mat->map_w, item.col0 + bx * 64, item.row0 + i * 128, bar);
-    };
-    auto load_s = [&](int c) {
-        const int s = c % cstages;
-        const uint32_t bar = ptx::smem_addr(&ctl->c_full[s]);
-        ptx::mbar_arrive_expect_tx(bar, S_CHUNK_BYTES);
-        ptx::tma_load_2d(c_ring + s * S_CHUNK_BYTES, &mat->map_s, (c % kchunks) * 32, item.row0 + (c / kchunks) * 128, bar);
-    };
-    if (warp == 0 && lane == 0) {
-        ptx::prefetch_tensormap(&mat->map_w);
-        for (int i = 0; i < min(slots, item.tiles); ++i) load_w(i);
-    } else if (warp == 6 && lane == 0) {
-        ptx::prefetch_tensormap(&mat->map_s);
-        for (int c = 0; c < min(cstages, total_chunks); ++c) load_s(c);
-    }
-    {
-        // slab of A as the N x K operand: row = column of W, K = index j of the sketch, values rounded to bf16
-        // and widened to 32 bits (exact in tf32).  One task makes a 4-column x 4-j block (four Philox blocks)
-        // and stores one 16-byte chunk per column; j >= r is written as zero.
-        const PhiloxKey key = make_key(seeds.s[item.mat - seed_base]);
-        const int jgroups = kchunks * 8;
-        const int tasks = (bn >> 2) * jgroups;
-        for (int t = threadIdx.x; t < tasks; t += K2_THREADS) {
-            const int jg = t % jgroups, cq = t / jgroups;
-            float v[4][4];
-#pragma unroll
-            for (int jj = 0; jj < 4; ++jj) {
-                float q[4] = {0.f, 0.f, 0.f, 0.f};
-                if (jg * 4 + jj < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)(jg * 4 + jj), key, scale, q);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) v[u][jj] = bf16_round(q[u]);
-            }
-            const uint32_t blk = slab + (jg >> 3) * slab_block;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int c = cq * 4 + u;
-                ptx::st_shared_v4(blk + c * 128 + (((jg & 7) ^ (c & 7)) << 4), __float_as_uint(v[u][0]), __float_as_uint(v[u][1]),
-                                  __float_as_uint(v[u][2]), __float_as_uint(v[u][3]));
-            }
-        }
-        ptx::fence_proxy_async_smem();
-    }
-    __syncthreads();
-
     if (warp == 0) {
-        // ------------------------------------------------------------------ W tile loads: refill slots as the stores free them
+        // ------------------------------------------------------------------ W tile loads
         if (lane == 0) {
-            int issued = min(slots, item.tiles);
-            for (int i = issued; i < item.tiles; ++i) {
-                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->w_free[i % slots]), ((i / slots) & 1) ^ 1, abort)) break;
-                load_w(i);
-                issued = i + 1;
+            int gt = 0, pending_from = 0;                       // tiles issued so far over all items of this CTA
+            bool ok = true;
+            for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+                const K2Item item = items[it];
+                const TcMatrix* mat = mats + item.mat;
+                const int live_boxes = min(boxes, (mat->m - item.col0 + 63) >> 6);
+                for (int i = 0; i < item.tiles; ++i, ++gt) {
+                    const int s = gt % slots;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->w_free[s]), ((gt / slots) & 1) ^ 1, abort);
+                    if (!ok) break;
+                    const uint32_t bar = ptx::smem_addr(&ctl->w_full[s]);
+                    ptx::mbar_arrive_expect_tx(bar, (uint32_t)live_boxes * W_BOX_BYTES);
+                    for (int bx = 0; bx < live_boxes; ++bx)
+                        ptx::tma_load_2d(w_ring + s * slot_bytes + bx * W_BOX_BYTES, &mat->map_w, item.col0 + bx * 64, item.row0 + i * 128, bar);
+                }
             }
-            if (*abort)   // loads that nobody consumed: wait (bounded) until they have landed
-                for (int i = max(0, issued - slots); i < issued; ++i)
-                    ptx::mbar_wait(ptx::smem_addr(&ctl->w_full[i % slots]), (i / slots) & 1, abort);
+            if (*abort) {   // loads that nobody consumed: wait (bounded) until they have landed
+                pending_from = max(0, gt - slots);
+                for (int g = pending_from; g < gt; ++g) ptx::mbar_wait(ptx::smem_addr(&ctl->w_full[g % slots]), (g / slots) & 1, abort);
+            }
         }
     } else if (warp == 6) {
         // ------------------------------------------------------------------ S chunk loads (fp32 rows, 32 columns each)
         if (lane == 0) {
-            int issued = min(cstages, total_chunks);
-            for (int c = issued; c < total_chunks; ++c) {
-                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->c_empty[c % cstages]), ((c / cstages) & 1) ^ 1, abort)) break;
-                load_s(c);
-                issued = c + 1;
+            int gc = 0;
+            bool ok = true;
+            for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+                const K2Item item = items[it];
+                const TcMatrix* mat = mats + item.mat;
+                for (int c = 0; c < item.tiles * kchunks; ++c, ++gc) {
+                    const int s = gc % cstages;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_empty[s]), ((gc / cstages) & 1) ^ 1, abort);
+                    if (!ok) break;
+                    const uint32_t bar = ptx::smem_addr(&ctl->c_full[s]);
+                    ptx::mbar_arrive_expect_tx(bar, S_CHUNK_BYTES);
+                    ptx::tma_load_2d(c_ring + s * S_CHUNK_BYTES, &mat->map_s, (c % kchunks) * 32, item.row0 + (c / kchunks) * 128, bar);
+                }
             }
             if (*abort)
-                for (int c = max(0, issued - cstages); c < issued; ++c)
-                    ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[c % cstages]), (c / cstages) & 1, abort);
+                for (int g = max(0, gc - cstages); g < gc; ++g) ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[g % cstages]), (g / cstages) & 1, abort);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc = ptx::umma_idesc_tf32((uint32_t)bn);
+            int gt = 0, gc = 0, k = 0;
             bool ok = true;
-            for (int i = 0; i < item.tiles && ok; ++i) {
-                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[i & 1]), ((i >> 1) & 1) ^ 1, abort);
-                for (int kc = 0; kc < kchunks && ok; ++kc) {
-                    const int c = i * kchunks + kc, s = c % cstages;
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[s]), (c / cstages) & 1, abort);
-                    if (!ok) break;
-                    ptx::tc_fence_after_sync();
+            for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++k) {
+                const K2Item item = items[it];
+                const uint32_t slab = slab0 + (k & 1) * slab_bytes;
+                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_full[k & 1]), (k >> 1) & 1, abort);
+                for (int i = 0; i < item.tiles && ok; ++i, ++gt) {
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[gt & 1]), ((gt >> 1) & 1) ^ 1, abort);
+                    for (int kc = 0; kc < kchunks && ok; ++kc, ++gc) {
+                        const int s = gc % cstages;
+                        ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[s]), (gc / cstages) & 1, abort);
+                        if (!ok) break;
+                        ptx::tc_fence_after_sync();
 #pragma unroll
-                    for (int k8 = 0; k8 < 4; ++k8)
-                        ptx::umma_tf32(tmem + (i & 1) * bn, ptx::umma_desc_k_sw128(c_ring + s * S_CHUNK_BYTES + k8 * 32),
-                                       ptx::umma_desc_k_sw128(slab + kc * slab_block + k8 * 32), idesc, (kc | k8) != 0);
-                    ptx::umma_commit(ptx::smem_addr(&ctl->c_empty[s]));
+                        for (int k8 = 0; k8 < 4; ++k8)
+                            ptx::umma_tf32(tmem + (gt & 1) * bn, ptx::umma_desc_k_sw128(c_ring + s * S_CHUNK_BYTES + k8 * 32),
+                                           ptx::umma_desc_k_sw128(slab + kc * slab_block + k8 * 32), idesc, (kc | k8) != 0);
+                        ptx::umma_commit(ptx::smem_addr(&ctl->c_empty[s]));
+                    }
+                    if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->acc_full[gt & 1]));
                 }
-                if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->acc_full[i & 1]));
+                if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->slab_empty[k & 1]));   // every MMA that reads this slab has completed
             }
         }
     } else if (warp == 7) {
         // ------------------------------------------------------------------ W tile stores
         if (lane == 0) {
-            for (int i = 0; i < item.tiles; ++i) {
-                const int s = i % slots;
-                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->out_ready[s]), (i / slots) & 1, abort)) break;
-                for (int bx = 0; bx < live_boxes; ++bx)
-                    ptx::tma_store_2d(&mat->map_w, item.col0 + bx * 64, item.row0 + i * 128, w_ring + s * slot_bytes + bx * W_BOX_BYTES);
-                ptx::tma_store_commit();
-                ptx::tma_store_wait_read<0>();              // the slot has been read out: it can be refilled
-                ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[s]));
+            int gt = 0;
+            bool ok = true;
+            for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+                const K2Item item = items[it];
+                const TcMatrix* mat = mats + item.mat;
+                const int live_boxes = min(boxes, (mat->m - item.col0 + 63) >> 6);
+                for (int i = 0; i < item.tiles; ++i, ++gt) {
+                    const int s = gt % slots;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->out_ready[s]), (gt / slots) & 1, abort);
+                    if (!ok) break;
+                    for (int bx = 0; bx < live_boxes; ++bx)
+                        ptx::tma_store_2d(&mat->map_w, item.col0 + bx * 64, item.row0 + i * 128, w_ring + s * slot_bytes + bx * W_BOX_BYTES);
+                    ptx::tma_store_commit();
+                    ptx::tma_store_wait_read<0>();              // the slot has been read out: it can be refilled
+                    ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[s]));
+                }
             }
             ptx::tma_store_wait_all<0>();
         }
     } else if (warp >= 2 && warp <= 5) {
         // ------------------------------------------------------------------ combine the accumulator with the W tile
         const int quarter = warp & 3;                          // tensor-memory lanes 32*quarter .. +31
+        const int row = quarter * 32 + lane;
+        int gt = 0;
         bool ok = true;
-        for (int i = 0; i < item.tiles && ok; ++i) {
-            const int s = i % slots;
-            ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[i & 1]), (i >> 1) & 1, abort) &&
-                 ptx::mbar_wait(ptx::smem_addr(&ctl->w_full[s]), (i / slots) & 1, abort);
-            if (!ok) break;
-            ptx::tc_fence_after_sync();
-            const int row = quarter * 32 + lane;
-            const uint32_t wrow = w_ring + s * slot_bytes + row * 128;
-            for (int c16 = 0; c16 < (live_boxes << 2); ++c16) {
-                uint32_t acc[16];
-                ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + (i & 1) * bn + c16 * 16, acc);
-                ptx::tmem_ld_wait();
-                const uint32_t box = wrow + (c16 >> 2) * W_BOX_BYTES;
+        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+            const K2Item item = items[it];
+            const int live_boxes = min(boxes, (mats[item.mat].m - item.col0 + 63) >> 6);
+            for (int i = 0; i < item.tiles; ++i, ++gt) {
+                const int s = gt % slots;
+                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[gt & 1]), (gt >> 1) & 1, abort) &&
+                     ptx::mbar_wait(ptx::smem_addr(&ctl->w_full[s]), (gt / slots) & 1, abort);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t wrow = w_ring + s * slot_bytes + row * 128;
+                for (int c16 = 0; c16 < (live_boxes << 2); ++c16) {
+                    uint32_t acc[16];
+                    ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + (gt & 1) * bn + c16 * 16, acc);
+                    ptx::tmem_ld_wait();
+                    const uint32_t box = wrow + (c16 >> 2) * W_BOX_BYTES;
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint32_t addr = box + (((((c16 & 3) << 1) + h) ^ (row & 7)) << 4);
-                    uint32_t x[4];
-                    ptx::ld_shared_v4(addr, x[0], x[1], x[2], x[3]);
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t addr = box + (((((c16 & 3) << 1) + h) ^ (row & 7)) << 4);
+                        uint32_t x[4];
+                        ptx::ld_shared_v4(addr, x[0], x[1], x[2], x[3]);
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const __nv_bfloat162 old = *reinterpret_cast<__nv_bfloat162*>(&x[u]);
-                        const float lo = fmaf(-step, __uint_as_float(acc[h * 8 + 2 * u]), __low2float(old));
-                        const float hi = fmaf(-step, __uint_as_float(acc[h * 8 + 2 * u + 1]), __high2float(old));
-                        __nv_bfloat162 nw = __floats2bfloat162_rn(lo, hi);
-                        x[u] = *reinterpret_cast<uint32_t*>(&nw);
+                        for (int u = 0; u < 4; ++u) {
+                            const __nv_bfloat162 old = *reinterpret_cast<__nv_bfloat162*>(&x[u]);
+                            const float lo = fmaf(-step, __uint_as_float(acc[h * 8 + 2 * u]), __low2float(old));
+                            const float hi = fmaf(-step, __uint_as_float(acc[h * 8 + 2 * u + 1]), __high2float(old));
+                            __nv_bfloat162 nw = __floats2bfloat162_rn(lo, hi);
+                            x[u] = *reinterpret_cast<uint32_t*>(&nw);
+                        }
+                        ptx::st_shared_v4(addr, x[0], x[1], x[2], x[3]);
                     }
-                    ptx::st_shared_v4(addr, x[0], x[1], x[2], x[3]);
+                }
+                ptx::tc_fence_before_sync();
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    ptx::mbar_arrive(ptx::smem_addr(&ctl->acc_empty[gt & 1]));
+                    ptx::mbar_arrive(ptx::smem_addr(&ctl->out_ready[s]));
                 }
             }
-            ptx::tc_fence_before_sync();
+        }
+    } else {
+        // ------------------------------------------------------------------ slab generators
+        // Slab of A as the N x K operand: row = column of W, K = index j of the sketch, values rounded to bf16
+        // and widened to 32 bits (exact in tf32).  One task makes a 4-column x 4-j block (four Philox blocks) and
+        // stores one 16-byte chunk per column; j >= r is written as zero.
+        const int g = threadIdx.x - 32 * K2_FIXED_WARPS;
+        const int jgroups = kchunks * 8;
+        const int tasks = (bn >> 2) * jgroups;
+        int k = 0;
+        bool ok = true;
+        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++k) {
+            const K2Item item = items[it];
+            const PhiloxKey key = make_key(seeds.s[item.mat - seed_base]);
+            ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_empty[k & 1]), ((k >> 1) & 1) ^ 1, abort);
+            if (!ok) break;
+            const uint32_t slab = slab0 + (k & 1) * slab_bytes;
+            for (int t = g; t < tasks; t += 32 * GW) {
+                const int jg = t % jgroups, cq = t / jgroups;
+                float v[4][4];
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    float q[4] = {0.f, 0.f, 0.f, 0.f};
+                    if (jg * 4 + jj < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)(jg * 4 + jj), key, scale, q);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) v[u][jj] = bf16_round(q[u]);
+                }
+                const uint32_t blk = slab + (jg >> 3) * slab_block;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int c = cq * 4 + u;
+                    ptx::st_shared_v4(blk + c * 128 + (((jg & 7) ^ (c & 7)) << 4), __float_as_uint(v[u][0]), __float_as_uint(v[u][1]),
+                                      __float_as_uint(v[u][2]), __float_as_uint(v[u][3]));
+                }
+            }
             ptx::fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) {
-                ptx::mbar_arrive(ptx::smem_addr(&ctl->acc_empty[i & 1]));
-                ptx::mbar_arrive(ptx::smem_addr(&ctl->out_ready[s]));
-            }
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->slab_full[k & 1]));
         }
     }
     ptx::tc_fence_before_sync();
@@ -575,7 +604,8 @@ struct TcSet {
     std::vector<int> k1_launch_begin;   // item ranges per launch (at most SEEDS_PER_LAUNCH matrices each)
     std::vector<int> split_mats;        // matrices whose sketch is updated by several items
     // decompression
-    int bn = 128, slots = 2, cstages = 2;
+    int bn = 128, slots = 2, cstages = 2, k2_gw = 8, k2_grid_max = 148;
+    std::vector<int> k2_launch_first_mat;
     size_t k2_smem = 0;
     K2Item* d_k2 = nullptr;
     std::vector<K2Item> h_k2;
@@ -842,55 +872,92 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
     set.k1_launch_begin.push_back((int)set.h_k1.size());
 }
 
-// Work decomposition of the decompression kernel: column slabs of bn columns, cut into runs of row tiles.
+// Work decomposition of the decompression kernel: column slabs of bn columns, cut into runs of row tiles; the
+// persistent CTAs take the items round-robin, largest first.
 inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
 {
     const int kchunks = (r + 31) / 32;
-    int bn = kchunks > 4 ? 64 : 128;
+    int bn = kchunks > 2 ? 64 : 128;
     bn = tune_knob("FLORA_K2_BN", bn, 64, 128) >= 128 ? 128 : 64;
     const size_t slab_bytes = (size_t)kchunks * bn * 128, slot = (size_t)(bn / 64) * W_BOX_BYTES, ctl = sizeof(K2Smem) + 1024;
-    // two CTAs per SM when two of them fit (each with two W slots and one S chunk): the fixed cost of one
-    // CTA (its slab) hides behind the streaming of the other
+    // two CTAs per SM when two of them fit (each with two slabs, two W slots and one S chunk)
     const size_t per_cta_max = 113 * 1024;                       // half of an SM's shared memory minus the reserve
-    int per_sm = (slab_bytes + S_CHUNK_BYTES + 2 * slot + ctl <= per_cta_max) ? 2 : 1;
+    int per_sm = (2 * slab_bytes + S_CHUNK_BYTES + 2 * slot + ctl <= per_cta_max) ? 2 : 1;
     per_sm = tune_knob("FLORA_K2_PER_SM", per_sm, 1, 2);
-    const size_t budget = (per_sm == 2 ? per_cta_max : SMEM_BUDGET) - ctl - slab_bytes;
+    const size_t budget = (per_sm == 2 ? per_cta_max : SMEM_BUDGET) - ctl - 2 * slab_bytes;
     int cstages = std::max(2, std::min(kchunks + 1, 4));
     cstages = tune_knob("FLORA_K2_CSTAGES", cstages, 1, K2_MAX_CSTAGES);
     while (cstages > 1 && (size_t)cstages * S_CHUNK_BYTES + 2 * slot > budget) --cstages;
     int slots = (int)std::min<size_t>(K2_MAX_SLOTS, (budget - (size_t)cstages * S_CHUNK_BYTES) / slot);
     slots = tune_knob("FLORA_K2_SLOTS", slots, 1, std::max(1, slots));
+    int GW = per_sm == 2 ? 4 : 8;
+    GW = tune_knob("FLORA_K2_GEN_WARPS", GW, 1, per_sm == 2 ? 4 : K2_MAX_GEN_WARPS);
     set.bn = bn;
     set.slots = slots;
     set.cstages = cstages;
-    set.k2_smem = slab_bytes + (size_t)cstages * S_CHUNK_BYTES + (size_t)slots * slot + sizeof(K2Smem) + 1024;
-    const int run = tune_knob("FLORA_K2_TILES", 8, 1, 1 << 20);      // row tiles per CTA, upper bound
-    set.h_k2.clear();
-    for (size_t i = 0; i < W.size(); ++i) {
-        const auto& w = W[i];
-        if (w.rows == 0 || w.cols == 0) continue;
-        const int64_t rtiles = (w.rows + 127) / 128, slabs = (w.cols + bn - 1) / bn;
-        const int64_t groups = (rtiles + run - 1) / run;
-        const int64_t per = (rtiles + groups - 1) / groups;
-        for (int64_t sl = 0; sl < slabs; ++sl)
-            for (int64_t t0 = 0; t0 < rtiles; t0 += per) {
-                K2Item it;
-                it.mat = (int)i;
-                it.col0 = (int)(sl * bn);
-                it.row0 = (int)(t0 * 128);
-                it.tiles = (int)std::min<int64_t>(per, rtiles - t0);
-                set.h_k2.push_back(it);
-            }
-    }
-    set.k2_launch_begin.clear();
-    int begin_mat = -1;
-    for (size_t k = 0; k < set.h_k2.size(); ++k) {
-        if (begin_mat < 0 || set.h_k2[k].mat >= begin_mat + SEEDS_PER_LAUNCH) {
-            begin_mat = set.h_k2[k].mat;
-            set.k2_launch_begin.push_back((int)k);
+    set.k2_gw = GW;
+    set.k2_smem = 2 * slab_bytes + (size_t)cstages * S_CHUNK_BYTES + (size_t)slots * slot + sizeof(K2Smem) + 1024;
+    const int grid_max = sm_count() * per_sm;
+    // cost model (microseconds of one SM): a tile streams bn*128*4 bytes at the SM's share of HBM; a slab costs
+    // r*bn normals at the generator warps' rate and overlaps the previous item's streaming
+    const double t_tile = (double)bn * 128 * 4 / (6.5e6 / sm_count()) ;
+    const double t_slab = (double)r * bn / (GW >= 8 ? 3200.0 : 2000.0) / per_sm;
+    auto build = [&](int run, std::vector<K2Item>& out) {
+        out.clear();
+        for (size_t i = 0; i < W.size(); ++i) {
+            const auto& w = W[i];
+            if (w.rows == 0 || w.cols == 0) continue;
+            const int64_t rtiles = (w.rows + 127) / 128, slabs = (w.cols + bn - 1) / bn;
+            const int64_t groups = (rtiles + run - 1) / run;
+            const int64_t per = (rtiles + groups - 1) / groups;
+            for (int64_t sl = 0; sl < slabs; ++sl)
+                for (int64_t t0 = 0; t0 < rtiles; t0 += per) {
+                    K2Item it;
+                    it.mat = (int)i;
+                    it.col0 = (int)(sl * bn);
+                    it.row0 = (int)(t0 * 128);
+                    it.tiles = (int)std::min<int64_t>(per, rtiles - t0);
+                    out.push_back(it);
+                }
+        }
+    };
+    auto sort_items = [&](std::vector<K2Item>& v, size_t b0, size_t b1) {
+        std::stable_sort(v.begin() + b0, v.begin() + b1, [](const K2Item& x, const K2Item& y) { return x.tiles > y.tiles; });
+    };
+    auto makespan = [&](const std::vector<K2Item>& v) {
+        const int grid = (int)std::min<size_t>(grid_max, v.size());
+        std::vector<K2Item> sorted = v;
+        sort_items(sorted, 0, sorted.size());
+        std::vector<double> t((size_t)std::max(grid, 1), 0.0);
+        for (size_t k = 0; k < sorted.size(); ++k) t[k % t.size()] += std::max(t_slab, sorted[k].tiles * t_tile * per_sm) + 0.2;
+        return *std::max_element(t.begin(), t.end());
+    };
+    const int fixed_run = tune_knob("FLORA_K2_TILES", 0, 0, 1 << 20);
+    std::vector<K2Item> cand;
+    double best = 1e300;
+    for (int run : {1 << 20, 48, 32, 24, 16, 12, 8, 6, 4, 3, 2}) {
+        if (fixed_run && run != (1 << 20)) continue;
+        build(fixed_run ? fixed_run : run, cand);
+        const double span = makespan(cand);
+        if (span < best * 0.97) {
+            best = span;
+            set.h_k2 = cand;
         }
     }
+    // launches cover at most SEEDS_PER_LAUNCH consecutive matrices; inside a launch the largest items go first
+    set.k2_launch_begin.clear();
+    set.k2_launch_first_mat.clear();
+    size_t u0 = 0;
+    while (u0 < set.h_k2.size()) {
+        size_t u1 = u0;
+        while (u1 < set.h_k2.size() && set.h_k2[u1].mat < set.h_k2[u0].mat + SEEDS_PER_LAUNCH) ++u1;
+        set.k2_launch_begin.push_back((int)u0);
+        set.k2_launch_first_mat.push_back(set.h_k2[u0].mat);
+        sort_items(set.h_k2, u0, u1);
+        u0 = u1;
+    }
     set.k2_launch_begin.push_back((int)set.h_k2.size());
+    set.k2_grid_max = grid_max;
 }
 
 inline void tc_set_free_stream(TcSet& s, cudaStream_t st)
@@ -1066,11 +1133,12 @@ inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float s
     for (size_t l = 0; l + 1 < set.k2_launch_begin.size(); ++l) {
         const int begin = set.k2_launch_begin[l], end = set.k2_launch_begin[l + 1];
         if (end == begin) continue;
-        const int seed_base = set.h_k2[begin].mat;
+        const int seed_base = set.k2_launch_first_mat[l];
         SeedTable table;
         for (int i = 0; i < SEEDS_PER_LAUNCH; ++i) table.s[i] = seed_base + i < set.count ? seeds[seed_base + i] : 0;
-        decompress_tc_kernel<<<end - begin, K2_THREADS, set.k2_smem, st>>>(set.d_mats, set.d_k2 + begin, table, seed_base, r, scale,
-                                                                           step, set.bn, set.slots, set.cstages);
+        const int grid = std::min(set.k2_grid_max, end - begin);
+        decompress_tc_kernel<<<grid, 32 * (K2_FIXED_WARPS + set.k2_gw), set.k2_smem, st>>>(
+            set.d_mats, set.d_k2 + begin, end - begin, table, seed_base, r, scale, step, set.bn, set.slots, set.cstages, set.k2_gw);
         launches.fetch_add(1, std::memory_order_relaxed);
     }
     return cudaPeekAtLastError() == cudaSuccess ? FLORA_OK : FLORA_ERR_CUDA;
