@@ -28,11 +28,14 @@ struct alignas(128) TcMatrix {
     CUtensorMap map_g;   // gradient G, box 64 columns x 128 rows, 128-byte swizzle
     CUtensorMap map_w;   // weight W, same box (loads and stores)
     CUtensorMap map_s;   // sketch S (fp32), box 32 columns x 128 rows, 128-byte swizzle
+    CUtensorMap map_sb;  // bf16 copy of S (scratch, n x k_pad), box 64 columns x 128 rows, 128-byte swizzle
+    __nv_bfloat16* Sb;   // the bf16 copy (used by the decompression kernel for ranks above 64)
     float* S;            // sketch, n x r fp32
     int64_t lds;
     int32_t n, m;
-    int32_t pad[26];
+    int32_t pad[24];
 };
+static_assert(sizeof(TcMatrix) % 128 == 0, "matrix records hold TMA descriptors");
 
 struct K1Item {          // one CTA of the compression kernel
     int32_t mat;         // index into the matrix table
@@ -329,6 +332,7 @@ struct K2Smem {
     int abort;
 };
 
+template <bool BF16S>
 __global__ void __launch_bounds__(K2_MAX_THREADS, 1)
 decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict__ items, int n_items,
                      const __grid_constant__ SeedTable seeds, int seed_base, int r, float scale, float step, int bn, int slots,
@@ -336,7 +340,8 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
-    const int kchunks = (r + 31) >> 5;                         // 32-deep K chunks (one 128-byte row of fp32 each)
+    // K chunks: one 128-byte row of S each (32 fp32 values, or 64 bf16 values when the bf16 copy of S is used)
+    const int kchunks = BF16S ? (r + 63) >> 6 : (r + 31) >> 5;
     const int boxes = bn >> 6;                                 // 64-column boxes per W tile
     const uint32_t slab_block = (uint32_t)bn * 128u;           // one K chunk of a slab
     const uint32_t slab_bytes = kchunks * slab_block;
@@ -416,7 +421,8 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
                     if (!ok) break;
                     const uint32_t bar = ptx::smem_addr(&ctl->c_full[s]);
                     ptx::mbar_arrive_expect_tx(bar, S_CHUNK_BYTES);
-                    ptx::tma_load_2d(c_ring + s * S_CHUNK_BYTES, &mat->map_s, (c % kchunks) * 32, item.row0 + (c / kchunks) * 128, bar);
+                    if (BF16S) ptx::tma_load_2d(c_ring + s * S_CHUNK_BYTES, &mat->map_sb, (c % kchunks) * 64, item.row0 + (c / kchunks) * 128, bar);
+                    else ptx::tma_load_2d(c_ring + s * S_CHUNK_BYTES, &mat->map_s, (c % kchunks) * 32, item.row0 + (c / kchunks) * 128, bar);
                 }
             }
             if (*abort)
@@ -425,7 +431,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = ptx::umma_idesc_tf32((uint32_t)bn);
+            const uint32_t idesc = BF16S ? ptx::umma_idesc_bf16((uint32_t)bn) : ptx::umma_idesc_tf32((uint32_t)bn);
             int gt = 0, gc = 0, k = 0;
             bool ok = true;
             for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++k) {
@@ -440,9 +446,12 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
                         if (!ok) break;
                         ptx::tc_fence_after_sync();
 #pragma unroll
-                        for (int k8 = 0; k8 < 4; ++k8)
-                            ptx::umma_tf32(tmem + (gt & 1) * bn, ptx::umma_desc_k_sw128(c_ring + s * S_CHUNK_BYTES + k8 * 32),
-                                           ptx::umma_desc_k_sw128(slab + kc * slab_block + k8 * 32), idesc, (kc | k8) != 0);
+                        for (int k8 = 0; k8 < 4; ++k8) {
+                            const uint64_t da = ptx::umma_desc_k_sw128(c_ring + s * S_CHUNK_BYTES + k8 * 32);
+                            const uint64_t db = ptx::umma_desc_k_sw128(slab + kc * slab_block + k8 * 32);
+                            if (BF16S) ptx::umma_bf16(tmem + (gt & 1) * bn, da, db, idesc, (kc | k8) != 0);
+                            else ptx::umma_tf32(tmem + (gt & 1) * bn, da, db, idesc, (kc | k8) != 0);
+                        }
                         ptx::umma_commit(ptx::smem_addr(&ctl->c_empty[s]));
                     }
                     if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->acc_full[gt & 1]));
@@ -535,21 +544,42 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
             if (!ok) break;
             const uint32_t slab = slab0 + (k & 1) * slab_bytes;
             for (int t = g; t < tasks; t += 32 * GW) {
-                const int jg = t % jgroups, cq = t / jgroups;
-                float v[4][4];
-#pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
-                    float q[4] = {0.f, 0.f, 0.f, 0.f};
-                    if (jg * 4 + jj < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)(jg * 4 + jj), key, scale, q);
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) v[u][jj] = bf16_round(q[u]);
-                }
+                const int jg = t % jgroups, cq = t / jgroups;       // jg: 16-byte chunk along K (4 tf32 or 8 bf16 values)
                 const uint32_t blk = slab + (jg >> 3) * slab_block;
+                if (BF16S) {
+                    uint32_t packed[4][4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int c = cq * 4 + u;
-                    ptx::st_shared_v4(blk + c * 128 + (((jg & 7) ^ (c & 7)) << 4), __float_as_uint(v[u][0]), __float_as_uint(v[u][1]),
-                                      __float_as_uint(v[u][2]), __float_as_uint(v[u][3]));
+                    for (int jj = 0; jj < 8; jj += 2) {
+                        float v0[4] = {0.f, 0.f, 0.f, 0.f}, v1[4] = {0.f, 0.f, 0.f, 0.f};
+                        const int j = jg * 8 + jj;
+                        if (j < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)j, key, scale, v0);
+                        if (j + 1 < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)(j + 1), key, scale, v1);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            __nv_bfloat162 pr = __floats2bfloat162_rn(v0[u], v1[u]);
+                            packed[u][jj >> 1] = *reinterpret_cast<uint32_t*>(&pr);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int c = cq * 4 + u;
+                        ptx::st_shared_v4(blk + c * 128 + (((jg & 7) ^ (c & 7)) << 4), packed[u][0], packed[u][1], packed[u][2], packed[u][3]);
+                    }
+                } else {
+                    float v[4][4];
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {
+                        float q[4] = {0.f, 0.f, 0.f, 0.f};
+                        if (jg * 4 + jj < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)(jg * 4 + jj), key, scale, q);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) v[u][jj] = bf16_round(q[u]);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int c = cq * 4 + u;
+                        ptx::st_shared_v4(blk + c * 128 + (((jg & 7) ^ (c & 7)) << 4), __float_as_uint(v[u][0]), __float_as_uint(v[u][1]),
+                                          __float_as_uint(v[u][2]), __float_as_uint(v[u][3]));
+                    }
                 }
             }
             ptx::fence_proxy_async_smem();
@@ -573,6 +603,22 @@ __global__ void scale_sketches_kernel(const TcMatrix* __restrict__ mats, const i
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
         float* p = mat->S + (t / r) * mat->lds + (t % r);
         *p = (b == 0.0f) ? 0.0f : *p * b;
+    }
+}
+
+// bf16 copy of every sketch of the table, n x k_pad with zero padding (the M x K operand of the decompression
+// kernel for ranks above 64); blockIdx.y = matrix, one thread per pair of columns.
+__global__ void sketch_to_bf16_kernel(const TcMatrix* __restrict__ mats, int r, int k_pad)
+{
+    const TcMatrix* mat = mats + blockIdx.y;
+    const int half = k_pad >> 1;
+    const int64_t total = (int64_t)mat->n * half;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = t / half;
+        const int j = (int)(t % half) * 2;
+        const float* src = mat->S + row * mat->lds;
+        const float a = j < r ? src[j] : 0.0f, b = j + 1 < r ? src[j + 1] : 0.0f;
+        reinterpret_cast<__nv_bfloat162*>(mat->Sb + row * k_pad)[j >> 1] = __floats2bfloat162_rn(a, b);
     }
 }
 
@@ -605,6 +651,8 @@ struct TcSet {
     std::vector<int> split_mats;        // matrices whose sketch is updated by several items
     // decompression
     int bn = 128, slots = 2, cstages = 2, k2_gw = 8, k2_grid_max = 148;
+    bool k2_bf16 = false;               // ranks above 64: the kernel reads a bf16 copy of the sketches
+    __nv_bfloat16* d_sb = nullptr;      // that copy (scratch owned by the set)
     std::vector<int> k2_launch_first_mat;
     size_t k2_smem = 0;
     K2Item* d_k2 = nullptr;
@@ -876,7 +924,12 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
 // persistent CTAs take the items round-robin, largest first.
 inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
 {
-    const int kchunks = (r + 31) / 32;
+    // ranks up to 64 read the fp32 sketch directly (tf32 MMA); above that the bytes of S that a CTA pulls per W
+    // tile exceed what shared memory can keep in flight, so a bf16 copy of S is made first (half the bytes,
+    // twice the K depth per 128-byte row) and the MMA runs in bf16
+    const bool bf16s = tune_knob("FLORA_K2_BF16S", r > 64 ? 1 : 0, 0, 1) != 0;
+    set.k2_bf16 = bf16s;
+    const int kchunks = bf16s ? (r + 63) / 64 : (r + 31) / 32;
     int bn = kchunks > 2 ? 64 : 128;
     bn = tune_knob("FLORA_K2_BN", bn, 64, 128) >= 128 ? 128 : 64;
     const size_t slab_bytes = (size_t)kchunks * bn * 128, slot = (size_t)(bn / 64) * W_BOX_BYTES, ctl = sizeof(K2Smem) + 1024;
@@ -901,7 +954,7 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
     // cost model (microseconds of one SM): a tile streams bn*128*4 bytes at the SM's share of HBM; a slab costs
     // r*bn normals at the generator warps' rate and overlaps the previous item's streaming
     const double t_tile = (double)bn * 128 * 4 / (6.5e6 / sm_count()) ;
-    const double t_slab = (double)r * bn / (GW >= 8 ? 3200.0 : 2000.0) / per_sm;
+    const double t_slab = (double)r * bn / (GW >= 8 ? 3200.0 : 2000.0) * per_sm;
     auto build = [&](int run, std::vector<K2Item>& out) {
         out.clear();
         for (size_t i = 0; i < W.size(); ++i) {
@@ -967,16 +1020,19 @@ inline void tc_set_free_stream(TcSet& s, cudaStream_t st)
         if (s.d_k1) cudaFreeAsync(s.d_k1, st);
         if (s.d_k2) cudaFreeAsync(s.d_k2, st);
         if (s.d_split) cudaFreeAsync(s.d_split, st);
+        if (s.d_sb) cudaFreeAsync(s.d_sb, st);
     } else {
         if (s.d_mats) cudaFree(s.d_mats);
         if (s.d_k1) cudaFree(s.d_k1);
         if (s.d_k2) cudaFree(s.d_k2);
         if (s.d_split) cudaFree(s.d_split);
+        if (s.d_sb) cudaFree(s.d_sb);
     }
     s.d_mats = nullptr;
     s.d_k1 = nullptr;
     s.d_k2 = nullptr;
     s.d_split = nullptr;
+    s.d_sb = nullptr;
     s.compress_ready = s.decompress_ready = false;
 }
 inline void tc_set_free(TcSet& s) { tc_set_free_stream(s, nullptr); }
@@ -1033,6 +1089,38 @@ inline flora_status tc_set_build_on(TcSet& set, const std::vector<flora_mat>& G,
     std::vector<flora_mat> none;
     flora_status rc = tc_fill_matrices(set, g_ok ? G : none, w_ok ? W : none, S);
     if (rc) return rc;
+    if (w_ok) {
+        plan_decompress(set, W, set.r);
+        if (set.k2_bf16) {
+            // scratch for the bf16 copies of the sketches: n x k_pad each, 1 KB aligned
+            const int k_pad = (set.r + 63) & ~63;
+            size_t total = 0;
+            std::vector<size_t> offset(S.size());
+            for (size_t i = 0; i < S.size(); ++i) {
+                offset[i] = total;
+                total += (((size_t)S[i].rows * k_pad * 2) + 1023) & ~(size_t)1023;
+            }
+            if (total) {
+                cudaError_t e = transient ? cudaMallocAsync((void**)&set.d_sb, total, st) : cudaMalloc((void**)&set.d_sb, total);
+                if (e != cudaSuccess) {
+                    cudaGetLastError();
+                    return FLORA_ERR_ALLOC;
+                }
+            }
+            for (size_t i = 0; i < S.size(); ++i) {
+                if (S[i].rows == 0) continue;
+                TcMatrix& tm = set.h_mats[i];
+                tm.Sb = reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<uint8_t*>(set.d_sb) + offset[i]);
+                flora_mat sb;
+                sb.data = tm.Sb;
+                sb.rows = S[i].rows;
+                sb.cols = k_pad;
+                sb.ld = k_pad;
+                sb.dtype = FLORA_BF16;
+                if (!make_map(&tm.map_sb, sb)) return FLORA_ERR_CUDA;
+            }
+        }
+    }
     rc = upload(&set.d_mats, set.h_mats, transient, st);
     if (rc) return rc;
     if (g_ok) {
@@ -1046,11 +1134,11 @@ inline flora_status tc_set_build_on(TcSet& set, const std::vector<flora_mat>& G,
         set.compress_ready = true;
     }
     if (w_ok) {
-        plan_decompress(set, W, set.r);
         rc = upload(&set.d_k2, set.h_k2, transient, st);
         if (rc) return rc;
-        if (cudaFuncSetAttribute(decompress_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)set.k2_smem) != cudaSuccess)
-            return FLORA_ERR_CUDA;
+        cudaError_t e = set.k2_bf16 ? cudaFuncSetAttribute(decompress_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)set.k2_smem)
+                                    : cudaFuncSetAttribute(decompress_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)set.k2_smem);
+        if (e != cudaSuccess) return FLORA_ERR_CUDA;
         set.decompress_ready = true;
     }
     return FLORA_OK;
@@ -1130,6 +1218,14 @@ inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float s
 {
     const int r = set.r;
     const float scale = 1.0f / sqrtf((float)r);
+    if (set.k2_bf16) {
+        const int k_pad = (r + 63) & ~63;
+        for (int begin = 0; begin < set.count; begin += 65535) {
+            dim3 grid(32, (unsigned)std::min(65535, set.count - begin));
+            sketch_to_bf16_kernel<<<grid, 256, 0, st>>>(set.d_mats + begin, r, k_pad);
+            launches.fetch_add(1, std::memory_order_relaxed);
+        }
+    }
     for (size_t l = 0; l + 1 < set.k2_launch_begin.size(); ++l) {
         const int begin = set.k2_launch_begin[l], end = set.k2_launch_begin[l + 1];
         if (end == begin) continue;
@@ -1137,8 +1233,12 @@ inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float s
         SeedTable table;
         for (int i = 0; i < SEEDS_PER_LAUNCH; ++i) table.s[i] = seed_base + i < set.count ? seeds[seed_base + i] : 0;
         const int grid = std::min(set.k2_grid_max, end - begin);
-        decompress_tc_kernel<<<grid, 32 * (K2_FIXED_WARPS + set.k2_gw), set.k2_smem, st>>>(
-            set.d_mats, set.d_k2 + begin, end - begin, table, seed_base, r, scale, step, set.bn, set.slots, set.cstages, set.k2_gw);
+        if (set.k2_bf16)
+            decompress_tc_kernel<true><<<grid, 32 * (K2_FIXED_WARPS + set.k2_gw), set.k2_smem, st>>>(
+                set.d_mats, set.d_k2 + begin, end - begin, table, seed_base, r, scale, step, set.bn, set.slots, set.cstages, set.k2_gw);
+        else
+            decompress_tc_kernel<false><<<grid, 32 * (K2_FIXED_WARPS + set.k2_gw), set.k2_smem, st>>>(
+                set.d_mats, set.d_k2 + begin, end - begin, table, seed_base, r, scale, step, set.bn, set.slots, set.cstages, set.k2_gw);
         launches.fetch_add(1, std::memory_order_relaxed);
     }
     return cudaPeekAtLastError() == cudaSuccess ? FLORA_OK : FLORA_ERR_CUDA;
