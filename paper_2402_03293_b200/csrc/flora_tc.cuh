@@ -464,6 +464,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         if (lane == 0) {
             int gt = 0;
             bool ok = true;
+            const bool lag = slots >= 4;               // with few slots, freeing a slot one tile late costs more than it gains
             for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
                 const K2Item item = items[it];
                 const TcMatrix* mat = mats + item.mat;
@@ -475,10 +476,18 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
                     for (int bx = 0; bx < live_boxes; ++bx)
                         ptx::tma_store_2d(&mat->map_w, item.col0 + bx * 64, item.row0 + i * 128, w_ring + s * slot_bytes + bx * W_BOX_BYTES);
                     ptx::tma_store_commit();
-                    ptx::tma_store_wait_read<0>();              // the slot has been read out: it can be refilled
-                    ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[s]));
+                    if (lag) {
+                        // one store stays in flight: wait until all but the newest have read their slot, free that one
+                        ptx::tma_store_wait_read<1>();
+                        if (gt > 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[(gt - 1) % slots]));
+                    } else {
+                        ptx::tma_store_wait_read<0>();          // the slot has been read out: it can be refilled
+                        ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[s]));
+                    }
                 }
             }
+            ptx::tma_store_wait_read<0>();
+            if (lag && gt > 0 && ok) ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[(gt - 1) % slots]));
             ptx::tma_store_wait_all<0>();
         }
     } else if (warp >= 2 && warp <= 5) {
@@ -1220,8 +1229,11 @@ inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float s
     const float scale = 1.0f / sqrtf((float)r);
     if (set.k2_bf16) {
         const int k_pad = (r + 63) & ~63;
+        int max_rows = 1;
+        for (const auto& tm : set.h_mats) max_rows = std::max(max_rows, tm.n);
+        const unsigned bx = (unsigned)std::min<int64_t>(1024, ((int64_t)max_rows * (k_pad / 2) + 1023) / 1024);   // ~4 pairs per thread
         for (int begin = 0; begin < set.count; begin += 65535) {
-            dim3 grid(32, (unsigned)std::min(65535, set.count - begin));
+            dim3 grid(bx, (unsigned)std::min(65535, set.count - begin));
             sketch_to_bf16_kernel<<<grid, 256, 0, st>>>(set.d_mats + begin, r, k_pad);
             launches.fetch_add(1, std::memory_order_relaxed);
         }
