@@ -317,7 +317,7 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
 // tile in shared memory and a TMA store writes the tile back.  W is read once and written once.
 // All rings (W slots, S chunks, accumulators, slabs) run across item boundaries.
 // ------------------------------------------------------------------------------------------------
-constexpr int K2_FIXED_WARPS = 8;   // warp 0: W loads, 1: MMA, 2-5: combine, 6: S loads, 7: W stores, 8..: slab generators
+constexpr int K2_FIXED_WARPS = 12;  // warp 0: W loads, 1: MMA, 2-5 and 8-11: combine, 6: S loads, 7: W stores, 12..: slab generators
 constexpr int K2_MAX_GEN_WARPS = 8;
 constexpr int K2_MAX_THREADS = 32 * (K2_FIXED_WARPS + K2_MAX_GEN_WARPS);
 constexpr int K2_MAX_SLOTS = 6;
@@ -357,7 +357,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         for (int s = 0; s < slots; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->w_full[s]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->w_free[s]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctl->out_ready[s]), 4);
+            ptx::mbar_init(ptx::smem_addr(&ctl->out_ready[s]), 8);
         }
         for (int s = 0; s < cstages; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->c_full[s]), 1);
@@ -365,7 +365,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         }
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->acc_full[s]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[s]), 4);
+            ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[s]), 8);
             ptx::mbar_init(ptx::smem_addr(&ctl->slab_full[s]), GW);
             ptx::mbar_init(ptx::smem_addr(&ctl->slab_empty[s]), 1);
         }
@@ -490,15 +490,22 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
             if (lag && gt > 0 && ok) ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[(gt - 1) % slots]));
             ptx::tma_store_wait_all<0>();
         }
-    } else if (warp >= 2 && warp <= 5) {
+    } else if ((warp >= 2 && warp <= 5) || (warp >= 8 && warp <= 11)) {
         // ------------------------------------------------------------------ combine the accumulator with the W tile
-        const int quarter = warp & 3;                          // tensor-memory lanes 32*quarter .. +31
+        // Eight warps: warp w owns tensor-memory lanes 32*(w%4) .. +31 (rows of the tile); warps 2-5 take the left
+        // half of the tile's columns, warps 8-11 the right half.  All accumulator loads of a warp are issued
+        // before the first is consumed.
+        const int quarter = warp & 3;
+        const int half = warp >= 8 ? 1 : 0;
         const int row = quarter * 32 + lane;
+        const int per_half = boxes << 1;                       // 16-column chunks per half: 2 (bn 64) or 4 (bn 128)
         int gt = 0;
         bool ok = true;
         for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
             const K2Item item = items[it];
-            const int live_boxes = min(boxes, (mats[item.mat].m - item.col0 + 63) >> 6);
+            const int live_chunks = min(boxes, (mats[item.mat].m - item.col0 + 63) >> 6) << 2;
+            const int c_begin = half * per_half;
+            const int mine = max(0, min(per_half, live_chunks - c_begin));
             for (int i = 0; i < item.tiles; ++i, ++gt) {
                 const int s = gt % slots;
                 ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[gt & 1]), (gt >> 1) & 1, abort) &&
@@ -506,25 +513,31 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t wrow = w_ring + s * slot_bytes + row * 128;
-                for (int c16 = 0; c16 < (live_boxes << 2); ++c16) {
-                    uint32_t acc[16];
-                    ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + (gt & 1) * bn + c16 * 16, acc);
-                    ptx::tmem_ld_wait();
-                    const uint32_t box = wrow + (c16 >> 2) * W_BOX_BYTES;
+                uint32_t acc[4][16];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const uint32_t addr = box + (((((c16 & 3) << 1) + h) ^ (row & 7)) << 4);
-                        uint32_t x[4];
-                        ptx::ld_shared_v4(addr, x[0], x[1], x[2], x[3]);
+                for (int k = 0; k < 4; ++k)
+                    if (k < mine) ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + (gt & 1) * bn + (c_begin + k) * 16, acc[k]);
+                ptx::tmem_ld_wait();
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const __nv_bfloat162 old = *reinterpret_cast<__nv_bfloat162*>(&x[u]);
-                            const float lo = fmaf(-step, __uint_as_float(acc[h * 8 + 2 * u]), __low2float(old));
-                            const float hi = fmaf(-step, __uint_as_float(acc[h * 8 + 2 * u + 1]), __high2float(old));
-                            __nv_bfloat162 nw = __floats2bfloat162_rn(lo, hi);
-                            x[u] = *reinterpret_cast<uint32_t*>(&nw);
+                for (int k = 0; k < 4; ++k) {
+                    if (k < mine) {
+                        const int c16 = c_begin + k;
+                        const uint32_t box = wrow + (c16 >> 2) * W_BOX_BYTES;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint32_t addr = box + (((((c16 & 3) << 1) + h) ^ (row & 7)) << 4);
+                            uint32_t x[4];
+                            ptx::ld_shared_v4(addr, x[0], x[1], x[2], x[3]);
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                const __nv_bfloat162 old = *reinterpret_cast<__nv_bfloat162*>(&x[u]);
+                                const float lo = fmaf(-step, __uint_as_float(acc[k][h * 8 + 2 * u]), __low2float(old));
+                                const float hi = fmaf(-step, __uint_as_float(acc[k][h * 8 + 2 * u + 1]), __high2float(old));
+                                __nv_bfloat162 nw = __floats2bfloat162_rn(lo, hi);
+                                x[u] = *reinterpret_cast<uint32_t*>(&nw);
+                            }
+                            ptx::st_shared_v4(addr, x[0], x[1], x[2], x[3]);
                         }
-                        ptx::st_shared_v4(addr, x[0], x[1], x[2], x[3]);
                     }
                 }
                 ptx::tc_fence_before_sync();
@@ -945,15 +958,15 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
     // two CTAs per SM when two of them fit (each with two slabs, two W slots and one S chunk)
     const size_t per_cta_max = 113 * 1024;                       // half of an SM's shared memory minus the reserve
     int per_sm = (2 * slab_bytes + S_CHUNK_BYTES + 2 * slot + ctl <= per_cta_max) ? 2 : 1;
-    per_sm = tune_knob("FLORA_K2_PER_SM", per_sm, 1, 2);
+    per_sm = 1;   // twelve fixed warps plus generators: one CTA per SM
     const size_t budget = (per_sm == 2 ? per_cta_max : SMEM_BUDGET) - ctl - 2 * slab_bytes;
     int cstages = std::max(2, std::min(kchunks + 1, 4));
     cstages = tune_knob("FLORA_K2_CSTAGES", cstages, 1, K2_MAX_CSTAGES);
     while (cstages > 1 && (size_t)cstages * S_CHUNK_BYTES + 2 * slot > budget) --cstages;
     int slots = (int)std::min<size_t>(K2_MAX_SLOTS, (budget - (size_t)cstages * S_CHUNK_BYTES) / slot);
     slots = tune_knob("FLORA_K2_SLOTS", slots, 1, std::max(1, slots));
-    int GW = per_sm == 2 ? 4 : 8;
-    GW = tune_knob("FLORA_K2_GEN_WARPS", GW, 1, per_sm == 2 ? 4 : K2_MAX_GEN_WARPS);
+    int GW = 8;
+    GW = tune_knob("FLORA_K2_GEN_WARPS", GW, 1, K2_MAX_GEN_WARPS);
     set.bn = bn;
     set.slots = slots;
     set.cstages = cstages;
