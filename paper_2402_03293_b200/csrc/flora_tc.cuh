@@ -188,6 +188,7 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc = ptx::umma_idesc_bf16((uint32_t)r_pad);
+            const uint64_t desc_base = ptx::umma_desc_k_sw128(smem_base);
             bool ok = true;
             for (int ks = 0; ks < item.ksteps && ok; ++ks) {
                 const int s = ks % stages, it = ks / stages;
@@ -196,14 +197,14 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
                             : ptx::mbar_wait(ptx::smem_addr(&ctl->full_a[s]), it & 1, abort));
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                const uint32_t stage = smem_base + s * stage_bytes;
-                const uint32_t a_tile = stage + T * G_TILE_BYTES;
+                // descriptors differ from the ring base only in the start-address field (16-byte units)
+                const uint64_t dstage = desc_base + (uint64_t)((s * stage_bytes) >> 4);
+                const uint64_t da_tile = dstage + (uint64_t)((T * G_TILE_BYTES) >> 4);
                 for (int t = 0; t < item.tiles; ++t) {
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        ptx::umma_bf16(tmem + t * r_pad, ptx::umma_desc_k_sw128(stage + t * G_TILE_BYTES + kk * 32),
-                                       ptx::umma_desc_k_sw128(a_tile + kk * 32), idesc, (ks | kk) != 0);
-                    }
+                    for (int kk = 0; kk < 4; ++kk)
+                        ptx::umma_bf16(tmem + t * r_pad, dstage + (uint64_t)((t * G_TILE_BYTES + kk * 32) >> 4), da_tile + (uint64_t)(kk * 2), idesc,
+                                       (ks | kk) != 0);
                 }
                 // the stage is free once every CTA of the cluster has consumed its copy of the A tile
                 const uint32_t ebar = ptx::smem_addr(&ctl->empty[s]);
@@ -432,13 +433,15 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc = BF16S ? ptx::umma_idesc_bf16((uint32_t)bn) : ptx::umma_idesc_tf32((uint32_t)bn);
+            const uint64_t desc_ring = ptx::umma_desc_k_sw128(c_ring);
             int gt = 0, gc = 0, k = 0;
             bool ok = true;
             for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++k) {
                 const K2Item item = items[it];
-                const uint32_t slab = slab0 + (k & 1) * slab_bytes;
+                const uint64_t desc_slab = ptx::umma_desc_k_sw128(slab0 + (k & 1) * slab_bytes);
                 ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_full[k & 1]), (k >> 1) & 1, abort);
                 for (int i = 0; i < item.tiles && ok; ++i, ++gt) {
+                    const uint32_t acc_addr = tmem + (gt & 1) * bn;
                     ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[gt & 1]), ((gt >> 1) & 1) ^ 1, abort);
                     for (int kc = 0; kc < kchunks && ok; ++kc, ++gc) {
                         const int s = gc % cstages;
@@ -447,10 +450,11 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
                         ptx::tc_fence_after_sync();
 #pragma unroll
                         for (int k8 = 0; k8 < 4; ++k8) {
-                            const uint64_t da = ptx::umma_desc_k_sw128(c_ring + s * S_CHUNK_BYTES + k8 * 32);
-                            const uint64_t db = ptx::umma_desc_k_sw128(slab + kc * slab_block + k8 * 32);
-                            if (BF16S) ptx::umma_bf16(tmem + (gt & 1) * bn, da, db, idesc, (kc | k8) != 0);
-                            else ptx::umma_tf32(tmem + (gt & 1) * bn, da, db, idesc, (kc | k8) != 0);
+                            // descriptors differ from the ring / slab base only in the start-address field (16-byte units)
+                            const uint64_t da = desc_ring + (uint64_t)((s * S_CHUNK_BYTES + k8 * 32) >> 4);
+                            const uint64_t db = desc_slab + (uint64_t)((kc * slab_block + k8 * 32) >> 4);
+                            if (BF16S) ptx::umma_bf16(acc_addr, da, db, idesc, (kc | k8) != 0);
+                            else ptx::umma_tf32(acc_addr, da, db, idesc, (kc | k8) != 0);
                         }
                         ptx::umma_commit(ptx::smem_addr(&ctl->c_empty[s]));
                     }
@@ -975,8 +979,10 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
     const int grid_max = sm_count() * per_sm;
     // cost model (microseconds of one SM): a tile streams bn*128*4 bytes at the SM's share of HBM; a slab costs
     // r*bn normals at the generator warps' rate and overlaps the previous item's streaming
-    const double t_tile = (double)bn * 128 * 4 / (6.5e6 / sm_count()) ;
-    const double t_slab = (double)r * bn / (GW >= 8 ? 3200.0 : 2000.0) * per_sm;
+    // (an SM takes in about 60 GB/s whatever the source: the chunks of S count like the W tile itself)
+    const double t_tile = std::max((double)bn * 128 * 4 / (6.5e6 / sm_count()),
+                                   ((double)bn * 128 * 2 + (double)kchunks * S_CHUNK_BYTES) / 60e3);
+    const double t_slab = (double)r * bn / (GW >= 8 ? 2000.0 : 1300.0);   // generator warps share the SM with the streaming warps
     auto build = [&](int run, std::vector<K2Item>& out) {
         out.clear();
         for (size_t i = 0; i < W.size(); ++i) {
@@ -1004,13 +1010,17 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
         std::vector<K2Item> sorted = v;
         sort_items(sorted, 0, sorted.size());
         std::vector<double> t((size_t)std::max(grid, 1), 0.0);
-        for (size_t k = 0; k < sorted.size(); ++k) t[k % t.size()] += std::max(t_slab, sorted[k].tiles * t_tile * per_sm) + 0.2;
+        for (size_t k = 0; k < sorted.size(); ++k) {
+            // generation overlaps the streaming of the previous item, but the two compete for issue slots
+            const double stream = sorted[k].tiles * t_tile;
+            t[k % t.size()] += std::max(t_slab, stream) + 0.35 * std::min(t_slab, stream) + 0.2;
+        }
         return *std::max_element(t.begin(), t.end());
     };
     const int fixed_run = tune_knob("FLORA_K2_TILES", 0, 0, 1 << 20);
     std::vector<K2Item> cand;
     double best = 1e300;
-    for (int run : {1 << 20, 48, 32, 24, 16, 12, 8, 6, 4, 3, 2}) {
+    for (int run : {1 << 20, 48, 32, 24, 16, 12, 11, 8, 6, 4, 3, 2}) {
         if (fixed_run && run != (1 << 20)) continue;
         build(fixed_run ? fixed_run : run, cand);
         const double span = makespan(cand);
