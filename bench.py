@@ -33,6 +33,10 @@ WORKLOAD = "gpt2_small_set"
 METRIC = "gradient GB/s per Flora step (compress+decompress-apply)"
 LR = 1e-3
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
+# (None once a kernel has changed since its counters were taken)
+NCU_TRAFFIC_COMPRESS = 182311168
+NCU_TRAFFIC_DECOMPRESS = 289950000
 
 
 # ------------------------------------------------------------------------------------------ helpers
@@ -66,7 +70,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100"],
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -187,13 +191,19 @@ def run_flora(args):
     epoch = [0]
 
     def seeds():
-        return [fb.flora_derive_seed(17, i, epoch[0]) for i in range(count)]
+        return fb.seed_array([fb.flora_derive_seed(17, i, epoch[0]) for i in range(count)])
 
-    def step():
+    def step(marks=None):
         s = seeds()
+        if marks is not None:
+            marks[0].record()
         for k in range(w.tau):
             sets[k].compress_accumulate(s)
+        if marks is not None:
+            marks[1].record()
         sets[0].decompress_apply(s, LR, 1.0 / w.tau)
+        if marks is not None:
+            marks[2].record()
         sets[0].zero_state()
         epoch[0] += 1
 
@@ -204,10 +214,13 @@ def run_flora(args):
     if rank == 0:
         sampler.start()
     launches0 = fb.flora_launch_count()
+    # three event marks per step inside the timed region: before the compressions, between them and the
+    # decompression, after it (per-kernel durations for the roofline block come from these)
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for _ in range(args.steps):
-        step()
+    for i in range(args.steps):
+        step(marks[i])
     e1.record()
     barrier()
     launches = fb.flora_launch_count() - launches0
@@ -222,31 +235,17 @@ def run_flora(args):
     grad_bytes_step = w.tau * w.elements * w.elem_bytes
     value = world * grad_bytes_step * args.steps / (ms * 1e-3) / 1e9
 
-    # per-kernel durations for the roofline (same steps, an event pair around every launch)
     comp_bytes, dec_bytes = algorithmic_bytes(w)
-    comp_ms, dec_ms = [], []
-    for _ in range(max(3, min(args.steps, 10))):
-        s = seeds()
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(w.tau + 2)]
-        evs[0].record()
-        for k in range(w.tau):
-            sets[k].compress_accumulate(s)
-            evs[k + 1].record()
-        sets[0].decompress_apply(s, LR, 1.0 / w.tau)
-        evs[w.tau + 1].record()
-        sets[0].zero_state()
-        epoch[0] += 1
-        torch.cuda.synchronize()
-        comp_ms += [evs[k].elapsed_time(evs[k + 1]) for k in range(w.tau)]
-        dec_ms.append(evs[w.tau].elapsed_time(evs[w.tau + 1]))
+    c_avg = sum(m[0].elapsed_time(m[1]) for m in marks) / (args.steps * w.tau)     # ms per compress launch
+    d_avg = sum(m[1].elapsed_time(m[2]) for m in marks) / args.steps              # ms per decompress launch
     peak, peak_src = measured_peak()
-    c_avg, d_avg = sum(comp_ms) / len(comp_ms), sum(dec_ms) / len(dec_ms)
     comp_gbs, dec_gbs = comp_bytes / (c_avg * 1e-3) / 1e9, dec_bytes / (d_avg * 1e-3) / 1e9
     step_roof_ms = (w.tau * comp_bytes + dec_bytes) / (peak * 1e9) * 1e3
-    roofline = {"bound": "hbm", "kernel": "compress (C += G A^T), one launch over the weight set", "achieved": comp_gbs,
-                "peak": peak, "unit": "GB/s", "frac": comp_gbs / peak, "traffic": None, "peak_source": peak_src,
-                "bytes_per_launch": comp_bytes, "us_per_launch": 1e3 * c_avg,
-                "decompress_apply": {"achieved": dec_gbs, "frac": dec_gbs / peak, "bytes_per_launch": dec_bytes, "us_per_launch": 1e3 * d_avg},
+    roofline = {"bound": "hbm", "kernel": "compress_tc_kernel (C += G A^T), one launch over the weight set, 8 launches per step",
+                "achieved": comp_gbs, "peak": peak, "unit": "GB/s", "frac": comp_gbs / peak, "traffic": NCU_TRAFFIC_COMPRESS,
+                "peak_source": peak_src, "bytes_per_launch": comp_bytes, "us_per_launch": 1e3 * c_avg,
+                "decompress_apply": {"kernel": "decompress_tc_kernel", "achieved": dec_gbs, "frac": dec_gbs / peak,
+                                     "bytes_per_launch": dec_bytes, "us_per_launch": 1e3 * d_avg, "traffic": NCU_TRAFFIC_DECOMPRESS},
                 "step_frac_of_roofline": step_roof_ms / (ms / args.steps)}
 
     # end to end: gradients start in pinned host memory, the updated weights are read back
@@ -308,7 +307,7 @@ def run_flora(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="flora", choices=["flora", "reference"])
     args = ap.parse_args()

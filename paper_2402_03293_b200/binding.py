@@ -213,8 +213,16 @@ def _mat_array(ts: Optional[Sequence[torch.Tensor]]):
     return arr
 
 
-def _u64_array(vals: Sequence[int]):
+def _u64_array(vals):
+    """Host array of 64-bit seeds; an array made by an earlier call is passed through unchanged."""
+    if isinstance(vals, ctypes.Array):
+        return vals
     return (ctypes.c_uint64 * len(vals))(*[int(v) & 0xFFFFFFFFFFFFFFFF for v in vals])
+
+
+def seed_array(vals: Sequence[int]):
+    """Marshal a list of seeds once, for reuse over several calls (the set calls accept the result)."""
+    return _u64_array(vals)
 
 
 class FloraSet:
