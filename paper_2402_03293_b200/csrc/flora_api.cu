@@ -16,6 +16,7 @@
 #include "flora_rng.cuh"
 #include "flora_simt.cuh"
 #include "flora_tc.cuh"
+#include "flora_gram.cuh"
 
 using namespace flora;
 
@@ -228,6 +229,11 @@ flora_status flora_transfer_axpby(flora_mat* dst, const flora_mat* src, int64_t 
     if (st) return st;
     if (dst->rows == 0) return FLORA_OK;
     const int r = (int)dst->cols;
+    if (operand == FLORA_BF16 && g_force_path.load() != 1) {
+        std::vector<GramJob> jobs(1);
+        jobs[0] = GramJob{nullptr, (float*)dst->data, (const float*)src->data, dst->ld, src->ld, (int32_t)dst->rows, (int32_t)m, seed_old, seed_new};
+        if (dst->rows <= 0x7FFFFFFF && m <= 0x7FFFFFFF) return transfer_tc(jobs, r, a, b, as_stream(stream), g_launches);
+    }
     float* T = nullptr;
     if (cudaMallocAsync((void**)&T, sizeof(float) * r * r, as_stream(stream)) != cudaSuccess) {
         cudaGetLastError();
@@ -385,6 +391,18 @@ flora_status flora_set_resample_transfer(flora_set* set, const uint64_t* seeds_o
     const int r = set->r;
     float* T = nullptr;
     if (set->S.empty()) return FLORA_OK;
+    bool all_bf16 = g_force_path.load() != 1;
+    for (const auto& g : big) all_bf16 = all_bf16 && g.dtype == FLORA_BF16 && g.cols <= 0x7FFFFFFF && g.rows <= 0x7FFFFFFF;
+    if (all_bf16) {
+        // one gram launch and one apply launch over the whole set
+        std::vector<GramJob> jobs;
+        for (size_t i = 0; i < set->S.size(); ++i) {
+            if (set->S[i].rows == 0) continue;
+            jobs.push_back(GramJob{nullptr, (float*)set->S[i].data, (const float*)set->S[i].data, set->S[i].ld, set->S[i].ld,
+                                   (int32_t)set->S[i].rows, (int32_t)big[i].cols, seeds_old[i], seeds_new[i]});
+        }
+        return transfer_tc(jobs, r, 1.0f, 0.0f, as_stream(stream), g_launches);
+    }
     if (cudaMallocAsync((void**)&T, sizeof(float) * r * r, as_stream(stream)) != cudaSuccess) {
         cudaGetLastError();
         return FLORA_ERR_ALLOC;

@@ -92,7 +92,8 @@ def test_decompress_apply(n, m, r, dtype, force_simt):
 
 
 @pytest.mark.parametrize("operand", ["f32", "bf16"])
-@pytest.mark.parametrize("n,m,r", [(1, 1, 1), (9, 33, 4), (100, 515, 32), (257, 1024, 64), (40, 300, 256)])
+@pytest.mark.parametrize("n,m,r", [(1, 1, 1), (9, 33, 4), (100, 515, 32), (257, 1024, 64), (40, 300, 256), (300, 11008, 200),
+                                   (64, 4097, 130), (1000, 64, 8), (33, 70, 17)])
 def test_transfer(n, m, r, operand):
     M0 = torch.randn(n, r, device=DEV)
     M = M0.clone()
