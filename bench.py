@@ -27,6 +27,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+from paper_2402_03293_b200 import replicas  # noqa: E402
 from paper_2402_03293_b200 import workloads as wl  # noqa: E402
 
 WORKLOAD = "gpt2_small_set"
@@ -224,16 +225,12 @@ def run_flora(args):
     e1.record()
     barrier()
     launches = fb.flora_launch_count() - launches0
-    ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
-    if dist:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
     if fb.flora_device_status() != 0:
         raise RuntimeError("a device-side wait timed out during the timed region")
     grad_bytes_step = w.tau * w.elements * w.elem_bytes
-    value = world * grad_bytes_step * args.steps / (ms * 1e-3) / 1e9
+    agg = replicas.aggregate_throughput(grad_bytes_step, args.steps, e0.elapsed_time(e1), dist, dev)
+    ms, value = agg["ms"], agg["gbs"]
 
     comp_bytes, dec_bytes = algorithmic_bytes(w)
     c_avg = sum(m[0].elapsed_time(m[1]) for m in marks) / (args.steps * w.tau)     # ms per compress launch
@@ -270,12 +267,8 @@ def run_flora(args):
         e2e_step()
     e1.record()
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    if dist:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e = {"value": world * grad_bytes_step * e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
+    e2e_agg = replicas.aggregate_throughput(grad_bytes_step, e2e_steps, e0.elapsed_time(e1), dist, dev)
+    e2e = {"value": e2e_agg["gbs"], "unit": "GB/s",
            "h2d_bytes_per_step": grad_bytes_step, "d2h_bytes_per_step": w.elements * w.elem_bytes, "steps": e2e_steps}
 
     cpu_baseline = None
