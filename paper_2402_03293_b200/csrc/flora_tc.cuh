@@ -1193,6 +1193,15 @@ inline flora_status tc_set_rebind(TcSet& set, const std::vector<flora_mat>& G, c
     return upload(&set.d_mats, set.h_mats, false, st);
 }
 
+// Blocks per matrix for the element-wise helper kernels (zero, scale): about four elements per thread of the
+// largest sketch.
+inline unsigned helper_blocks(const TcSet& set)
+{
+    int64_t most = 1;
+    for (const auto& tm : set.h_mats) most = std::max<int64_t>(most, (int64_t)tm.n * set.r);
+    return (unsigned)std::min<int64_t>(1024, (most + 1023) / 1024);
+}
+
 inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, float b, cudaStream_t st,
                                     std::atomic<uint64_t>& launches)
 {
@@ -1201,7 +1210,7 @@ inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, 
     if (b != 1.0f && !set.split_mats.empty()) {
         // rows updated by several CTAs receive atomic adds: scale them by b first
         for (size_t begin = 0; begin < set.split_mats.size(); begin += 65535) {
-            dim3 grid(16, (unsigned)std::min<size_t>(65535, set.split_mats.size() - begin));
+            dim3 grid(helper_blocks(set), (unsigned)std::min<size_t>(65535, set.split_mats.size() - begin));
             scale_sketches_kernel<<<grid, 256, 0, st>>>(set.d_mats, set.d_split + begin, r, b);
             launches.fetch_add(1, std::memory_order_relaxed);
         }
@@ -1298,7 +1307,7 @@ inline bool tc_decompress_supported(const flora_mat* big, const flora_mat* sketc
 inline flora_status tc_set_zero(TcSet& set, cudaStream_t st, std::atomic<uint64_t>& launches)
 {
     for (int begin = 0; begin < set.count; begin += 65535) {
-        dim3 grid(32, (unsigned)std::min(65535, set.count - begin));
+        dim3 grid(helper_blocks(set), (unsigned)std::min(65535, set.count - begin));
         zero_sketches_kernel<<<grid, 256, 0, st>>>(set.d_mats + begin, set.r);
         launches.fetch_add(1, std::memory_order_relaxed);
     }
