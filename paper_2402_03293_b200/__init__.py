@@ -4,4 +4,4 @@ The CUDA library is loaded lazily by :mod:`paper_2402_03293_b200.binding`; impor
 package itself needs no GPU.  There is no CPU fallback: calling an operation without the
 built CUDA library raises.
 """
-__all__ = ["binding", "workloads", "hostlogic"]
+__all__ = ["binding", "workloads", "hostlogic", "replicas"]
