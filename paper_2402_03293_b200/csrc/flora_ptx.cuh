@@ -148,6 +148,14 @@ __device__ __forceinline__ void bulk_copy_to_peer(uint32_t dst_cluster_addr, uin
                  : "memory");
 }
 
+// ---------------------------------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-stream-serialization attribute may start while the previous kernel of
+// the stream is still running.  grid_dependency_wait() blocks until that kernel has completed and its writes are
+// visible; it must precede the first access to anything an earlier kernel may have written.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream begin its own set-up as soon as resources free up.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem()
 {

@@ -124,7 +124,8 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
     K1Smem* ctl = reinterpret_cast<K1Smem*>(smem_raw + (smem_base - ptx::smem_addr(smem_raw)) + (size_t)stages * stage_bytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    const K1Item item = items[blockIdx.x];
+    ptx::grid_launch_dependents();
+    const K1Item item = items[blockIdx.x];                    // tables and descriptors are written at set creation, not by kernels
     const TcMatrix* mat = mats + item.mat;
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < T * r_pad) tmem_cols <<= 1;
@@ -157,6 +158,9 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
     __syncthreads();
     if (S > 1) ptx::cluster_sync();       // every CTA's barriers exist before anyone arrives on them remotely
     ptx::tc_fence_after_sync();
+    // everything above touched only this CTA's shared and tensor memory; G and S may have been written by the
+    // previous kernel of the stream
+    ptx::grid_dependency_wait();
     const uint32_t tmem = ctl->tmem_base;
     volatile int* abort = &ctl->abort;
     const uint32_t rank = S > 1 ? ptx::cluster_ctarank() : 0u;
@@ -808,7 +812,7 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
     uint32_t cols = 32;
     while ((int)cols < T * r_pad) cols <<= 1;
     // cluster size from the generation / load ratio
-    const double ratio = r * 0.0305 / T;
+    const double ratio = r * 0.045 / T;
     int S = 1;
     while (S < 8 && ratio / S > 0.5) S <<= 1;
     while (S > 1 && (int64_t)S * T > 2 * max_tiles) S >>= 1;         // not more CTAs than there are rows to share
@@ -1226,13 +1230,15 @@ inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, 
         cfg.blockDim = dim3((unsigned)k1_threads(set.GW));
         cfg.dynamicSmemBytes = set.k1_smem;
         cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = (unsigned)set.S;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // the kernel waits for its predecessor itself
+        attr[0].val.programmaticStreamSerializationAllowed = tune_knob("FLORA_PDL", 1, 0, 1);
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)set.S;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = set.S > 1 ? 1 : 0;
+        cfg.numAttrs = set.S > 1 ? 2 : 1;
         const TcMatrix* mats = set.d_mats;
         const K1Item* items = set.d_k1 + begin;
         if (cudaLaunchKernelEx(&cfg, compress_tc_kernel, mats, items, table, seed_base, r, scale, a, b, set.T, set.stages, set.S, set.GW) !=
