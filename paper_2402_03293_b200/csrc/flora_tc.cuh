@@ -114,7 +114,7 @@ __device__ __forceinline__ void k1_store_chunk(float* srow, const uint32_t (&v)[
 
 __global__ void __launch_bounds__(K1_MAX_THREADS, 1)
 compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__ items, const __grid_constant__ SeedTable seeds,
-                   int seed_base, int r, float scale, float a, float b, int T, int stages, int S, int GW)
+                   int seed_base, int r, float scale, float a, float b, int T, int stages, int S, int GW, int late_wait)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
@@ -159,8 +159,9 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
     if (S > 1) ptx::cluster_sync();       // every CTA's barriers exist before anyone arrives on them remotely
     ptx::tc_fence_after_sync();
     // everything above touched only this CTA's shared and tensor memory; G and S may have been written by the
-    // previous kernel of the stream
-    ptx::grid_dependency_wait();
+    // previous kernel of the stream.  `late_wait`: that kernel is this library's own pre-scaling of S, which was
+    // itself ordered after everything before it and does not touch G, so only the accesses to S need to wait
+    if (!late_wait) ptx::grid_dependency_wait();
     const uint32_t tmem = ctl->tmem_base;
     volatile int* abort = &ctl->abort;
     const uint32_t rank = S > 1 ? ptx::cluster_ctarank() : 0u;
@@ -279,6 +280,7 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
             const int quarter = warp & 3;
             if (ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full), 0, abort)) {
                 ptx::tc_fence_after_sync();
+                if (late_wait) ptx::grid_dependency_wait();
                 const bool vec_ok = ((mat->lds & 3) == 0) && ((reinterpret_cast<uintptr_t>(mat->S) & 15) == 0);
                 // S <- S + a*acc needs no read; a split item adds into rows that were scaled by b beforehand
                 const bool add_only = item.direct == 0 || b == 1.0f;
@@ -286,16 +288,28 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
                     const int64_t row = (int64_t)item.row0 + t * 128 + quarter * 32 + lane;
                     const bool live = row < mat->n;
                     float* srow = mat->S + row * mat->lds;
-                    for (int j0 = 0; j0 < r_pad; j0 += 16) {
-                        float4 old[4] = {};
-                        if (live && !add_only && b != 0.0f && vec_ok && j0 + 16 <= r) {
+                    // the owner of a row reads its old values 32 columns at a time before the accumulator is fetched,
+                    // so the eight loads are in flight together
+                    const bool rmw = live && !add_only && b != 0.0f && vec_ok;
+                    for (int j32 = 0; j32 < r_pad; j32 += 32) {
+                        float4 old[2][4] = {};
+                        if (rmw) {
 #pragma unroll
-                            for (int u = 0; u < 4; ++u) old[u] = *reinterpret_cast<const float4*>(srow + j0 + 4 * u);
+                            for (int q = 0; q < 2; ++q)
+#pragma unroll
+                                for (int u = 0; u < 4; ++u)
+                                    if (j32 + 16 * q + 4 * u + 4 <= r) old[q][u] = *reinterpret_cast<const float4*>(srow + j32 + 16 * q + 4 * u);
                         }
-                        uint32_t v[16];
-                        ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + t * r_pad + j0, v);
-                        ptx::tmem_ld_wait();
-                        if (live) k1_store_chunk(srow, v, old, j0, r, a, b, add_only, vec_ok);
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            const int j0 = j32 + 16 * q;
+                            if (j0 < r_pad) {
+                                uint32_t v[16];
+                                ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + t * r_pad + j0, v);
+                                ptx::tmem_ld_wait();
+                                if (live) k1_store_chunk(srow, v, old[q], j0, r, a, b, add_only, vec_ok);
+                            }
+                        }
                     }
                 }
             }
@@ -628,6 +642,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
 // S <- b S for the listed matrices (those whose rows receive atomic adds from several CTAs); blockIdx.y = list entry.
 __global__ void scale_sketches_kernel(const TcMatrix* __restrict__ mats, const int* __restrict__ ids, int r, float b)
 {
+    ptx::grid_launch_dependents();       // the compression kernel that follows may start streaming G right away
     const TcMatrix* mat = mats + ids[blockIdx.y];
     const int64_t total = (int64_t)mat->n * r;
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
@@ -911,6 +926,15 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
                 units = cand_units;
                 set.split_mats = cand_split;
             }
+        }
+    }
+    // a schedule without any split over columns is preferred when it is nearly as short: every row of a sketch then
+    // has one owner, so a momentum update needs neither the pre-scaling pass nor atomic adds
+    if (!fixed_waves) {
+        build_units((int64_t)1 << 60, cand_units, cand_split);
+        if (makespan(cand_units) <= 1.12 * best_span) {
+            units = cand_units;
+            set.split_mats = cand_split;
         }
     }
     // launches cover at most SEEDS_PER_LAUNCH consecutive matrices; inside a launch the largest units go first
@@ -1211,10 +1235,14 @@ inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, 
 {
     const int r = set.r;
     const float scale = 1.0f / sqrtf((float)r);
+    int late_wait = 0;
     if (b != 1.0f && !set.split_mats.empty()) {
+        late_wait = tune_knob("FLORA_PDL", 1, 0, 1);
         // rows updated by several CTAs receive atomic adds: scale them by b first
         for (size_t begin = 0; begin < set.split_mats.size(); begin += 65535) {
-            dim3 grid(helper_blocks(set), (unsigned)std::min<size_t>(65535, set.split_mats.size() - begin));
+            const size_t jobs_here = std::min<size_t>(65535, set.split_mats.size() - begin);
+            // few enough blocks to be resident at once: the compression kernel may only start once all have started
+            dim3 grid((unsigned)std::max<size_t>(1, std::min<size_t>(helper_blocks(set), (size_t)sm_count() * 6 / jobs_here)), (unsigned)jobs_here);
             scale_sketches_kernel<<<grid, 256, 0, st>>>(set.d_mats, set.d_split + begin, r, b);
             launches.fetch_add(1, std::memory_order_relaxed);
         }
@@ -1241,7 +1269,7 @@ inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, 
         cfg.numAttrs = set.S > 1 ? 2 : 1;
         const TcMatrix* mats = set.d_mats;
         const K1Item* items = set.d_k1 + begin;
-        if (cudaLaunchKernelEx(&cfg, compress_tc_kernel, mats, items, table, seed_base, r, scale, a, b, set.T, set.stages, set.S, set.GW) !=
+        if (cudaLaunchKernelEx(&cfg, compress_tc_kernel, mats, items, table, seed_base, r, scale, a, b, set.T, set.stages, set.S, set.GW, l == 0 ? late_wait : 0) !=
             cudaSuccess)
             return FLORA_ERR_CUDA;
         launches.fetch_add(1, std::memory_order_relaxed);
