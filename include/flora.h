@@ -188,6 +188,11 @@ uint64_t flora_launch_count(void);
 /* Reads (synchronously, with a device->host copy) and clears the device-side error word that
  * bounded waits inside the kernels set when they give up: FLORA_OK or FLORA_ERR_TIMEOUT. */
 flora_status flora_device_status(void);
+/* Test hook for the bounded device-side waits: launches one small kernel whose only wait (limit 1 ms) can
+ * never be satisfied, synchronises `stream` and returns FLORA_ERR_TIMEOUT if the wait gave up as designed
+ * (FLORA_OK would mean it did not).  The device error word is raised as by a real timeout, so the next
+ * flora_device_status() also reports FLORA_ERR_TIMEOUT, once.  The context stays usable. */
+flora_status flora_debug_wait_timeout_selftest(void* stream);
 const char* flora_status_string(flora_status s);
 int flora_version(void);
 

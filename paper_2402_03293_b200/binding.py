@@ -29,7 +29,7 @@ EXPORTS = [
     "flora_set_rebind_gradients", "flora_set_compress_accumulate", "flora_set_momentum_step",
     "flora_set_decompress_apply", "flora_set_resample_transfer", "flora_set_zero_state", "flora_derive_seed",
     "flora_resamples_at", "flora_set_compress_accumulate_from_host", "flora_set_read_weights_to_host",
-    "flora_debug_force_path", "flora_launch_count", "flora_device_status", "flora_status_string", "flora_version",
+    "flora_debug_force_path", "flora_debug_wait_timeout_selftest", "flora_launch_count", "flora_device_status", "flora_status_string", "flora_version",
 ]
 
 
@@ -77,6 +77,7 @@ def load() -> ctypes.CDLL:
             "flora_set_compress_accumulate_from_host": (I32, [P, ctypes.POINTER(P), ctypes.POINTER(U64), P]),
             "flora_set_read_weights_to_host": (I32, [P, ctypes.POINTER(P), P]),
             "flora_debug_force_path": (None, [ctypes.c_int]),
+            "flora_debug_wait_timeout_selftest": (I32, [P]),
             "flora_launch_count": (U64, []),
             "flora_device_status": (I32, []),
             "flora_status_string": (ctypes.c_char_p, [I32]),
@@ -189,6 +190,11 @@ def flora_resamples_at(t: int, kappa: int) -> bool:
 
 def flora_debug_force_path(path: int) -> None:
     load().flora_debug_force_path(path)
+
+
+def flora_debug_wait_timeout_selftest(stream=None) -> int:
+    """Status of the bounded-wait self-test: FLORA_ERR_TIMEOUT (7) when the wait gave up as designed."""
+    return int(load().flora_debug_wait_timeout_selftest(_stream(stream)))
 
 
 def flora_launch_count() -> int:

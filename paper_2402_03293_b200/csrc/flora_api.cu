@@ -488,6 +488,24 @@ flora_status flora_device_status(void)
     return word ? FLORA_ERR_TIMEOUT : FLORA_OK;
 }
 
+flora_status flora_debug_wait_timeout_selftest(void* stream)
+{
+    int* flag = nullptr;
+    if (cudaMallocAsync((void**)&flag, sizeof(int), as_stream(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return FLORA_ERR_ALLOC;
+    }
+    cudaMemsetAsync(flag, 0, sizeof(int), as_stream(stream));
+    wait_timeout_selftest_kernel<<<1, 32, 0, as_stream(stream)>>>(flag);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    int gave_up = 0;
+    cudaError_t e = cudaMemcpyAsync(&gave_up, flag, sizeof(int), cudaMemcpyDeviceToHost, as_stream(stream));
+    if (e == cudaSuccess) e = cudaStreamSynchronize(as_stream(stream));
+    cudaFreeAsync(flag, as_stream(stream));
+    if (e != cudaSuccess) return FLORA_ERR_CUDA;
+    return gave_up ? FLORA_ERR_TIMEOUT : FLORA_OK;
+}
+
 const char* flora_status_string(flora_status s)
 {
     switch (s) {

@@ -1348,6 +1348,21 @@ inline flora_status tc_set_zero(TcSet& set, cudaStream_t st, std::atomic<uint64_
     return cudaPeekAtLastError() == cudaSuccess ? FLORA_OK : FLORA_ERR_CUDA;
 }
 
+// Self-test of the bounded waits: one CTA waits on a barrier that nothing ever arrives on, with a one-millisecond
+// limit.  The wait gives up, raises the error word and the kernel returns normally.
+__global__ void wait_timeout_selftest_kernel(int* gave_up)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_addr(&bar), 1);
+        abort_flag = 0;
+        ptx::fence_barrier_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) *gave_up = ptx::mbar_wait(ptx::smem_addr(&bar), 0, &abort_flag, 1000000ull) ? 0 : 1;
+}
+
 inline bool tc_read_and_clear_error(int* word)
 {
     int zero = 0;

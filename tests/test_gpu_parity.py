@@ -273,3 +273,39 @@ def test_full_size_set_sampled_rows(name):
         ref = oracle_decompress(W0[i][torch.from_numpy(rows).to(DEV)].cpu(), torch.from_numpy(got), seeds[i], 4.0, 0.5)
         assert rel_err(values(wl.as_numpy(W[i])[rows]), values(ref)) <= TOL["bf16"], i
     fset.close()
+
+
+# --------------------------------------------------------------------------------------- robustness
+def test_more_matrices_than_one_launch_carries_seeds_for():
+    """460 matrices: the set is cut into two launches (seeds travel as a kernel parameter, 448 per launch)."""
+    count, n, m, r = 460, 128, 128, 16
+    torch.manual_seed(1)
+    Gbig = (torch.randn(count, n, m, device=DEV) * 0.03).to(torch.bfloat16)
+    Wbig = (torch.randn(count, n, m, device=DEV) * 0.02).to(torch.bfloat16)
+    Sbig = torch.zeros(count, n, r, device=DEV)
+    G, W, S = [Gbig[i] for i in range(count)], [Wbig[i] for i in range(count)], [Sbig[i] for i in range(count)]
+    W0 = Wbig.clone()
+    fset = fb.FloraSet(G, W, S)
+    seeds = [fb.flora_derive_seed(2, i, 0) for i in range(count)]
+    fset.compress_accumulate(seeds)
+    fset.momentum_step(0.5, seeds)
+    fset.decompress_apply(seeds, 2.0, 1.0)
+    torch.cuda.synchronize()
+    for i in (0, 1, 447, 448, 449, 459):
+        c1 = oracle_compress(G[i], torch.zeros(n, r), seeds[i])
+        c2 = oracle_compress(G[i], torch.from_numpy(c1), seeds[i], a=0.5, b=0.5)
+        assert rel_err(S[i].cpu().numpy(), c2) <= TOL["bf16"], i
+        ref = oracle_decompress(W0[i], S[i], seeds[i], 2.0, 1.0)
+        assert rel_err(values(wl.as_numpy(W[i])), values(ref)) <= TOL["bf16"], i
+    fset.close()
+
+
+def test_bounded_wait_gives_up_and_reports_a_timeout():
+    """A wait that can never be satisfied returns after its limit, the status says so, and the device keeps working."""
+    assert fb.flora_debug_wait_timeout_selftest() == 7                 # FLORA_ERR_TIMEOUT
+    assert fb.flora_device_status() == 7                               # the error word was raised ...
+    assert fb.flora_device_status() == 0                               # ... and reading it cleared it
+    C = torch.zeros(256, 8, device=DEV)
+    G = _g(256, 512, "bf16", 3)
+    fb.flora_compress_accumulate(G, C, 5, 8)
+    assert rel_err(C.cpu().numpy(), oracle_compress(G, torch.zeros(256, 8), 5)) <= TOL["bf16"]
