@@ -181,7 +181,19 @@ __device__ __forceinline__ void tma_store_2d(const void* tmap, int x, int y, uin
                  ::"l"(tmap), "r"(src), "r"(x), "r"(y)
                  : "memory");
 }
+// The same, adding the tile element-wise (fp32, atomically per element) to what global memory holds.
+__device__ __forceinline__ void tma_reduce_add_2d(const void* tmap, int x, int y, uint32_t src)
+{
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(tmap), "r"(src), "r"(x), "r"(y)
+                 : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Barrier among `nthreads` threads (a multiple of 32) of the CTA that all name the same id (1..15; 0 is __syncthreads).
+__device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t nthreads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
 template <int N>
 __device__ __forceinline__ void tma_store_wait_read()
 {

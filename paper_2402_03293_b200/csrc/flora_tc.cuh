@@ -72,45 +72,14 @@ constexpr int K1_MAX_THREADS = 64 + 32 * K1_MAX_GEN_WARPS + 32;
 // threads of a CTA: producer warp, MMA warp, GW generator warps, one warp that forwards slices to cluster peers
 inline int k1_threads(int gen_warps) { return 64 + 32 * gen_warps + 32; }
 constexpr int G_TILE_BYTES = 128 * 128;   // 128 rows x 64 bf16
+constexpr int S_CHUNK_BYTES_K1 = 128 * 128; // 128 rows x 32 fp32
 
 struct K1Smem {                            // barriers and scalars, placed after the tile ring
-    uint64_t full_g[8], full_a[8], slice_ready[8], empty[8], acc_full;
+    uint64_t full_g[8], full_a[8], slice_ready[8], empty[8], acc_full, old_full[16];
     uint32_t tmem_base;
     int abort;
+    int epi_go[4];
 };
-
-// One row of one tile: sixteen accumulator columns j0..j0+15 into S.  `add_only`: S <- S + a*acc by atomic
-// adds (nothing is read back, so no memory latency sits on the critical path); otherwise the owner of the
-// row computes b*S + a*acc from values `old` that were loaded beforehand.
-__device__ __forceinline__ void k1_store_chunk(float* srow, const uint32_t (&v)[16], const float4 (&old)[4], int j0, int r, float a,
-                                               float b, bool add_only, bool vec_ok)
-{
-    if (vec_ok && j0 + 16 <= r) {
-#pragma unroll
-        for (int u = 0; u < 16; u += 4) {
-            const float x0 = a * __uint_as_float(v[u]), x1 = a * __uint_as_float(v[u + 1]);
-            const float x2 = a * __uint_as_float(v[u + 2]), x3 = a * __uint_as_float(v[u + 3]);
-            if (add_only) {
-                ptx::red_add_v4(srow + j0 + u, x0, x1, x2, x3);
-            } else {
-                const float4 o = old[u >> 2];
-                *reinterpret_cast<float4*>(srow + j0 + u) =
-                    (b == 0.0f) ? make_float4(x0, x1, x2, x3)
-                                : make_float4(fmaf(b, o.x, x0), fmaf(b, o.y, x1), fmaf(b, o.z, x2), fmaf(b, o.w, x3));
-            }
-        }
-    } else {
-#pragma unroll
-        for (int u = 0; u < 16; ++u) {
-            if (j0 + u < r) {
-                const float x = a * __uint_as_float(v[u]);
-                float* p = srow + j0 + u;
-                if (add_only) atomicAdd(p, x);
-                else *p = (b == 0.0f) ? x : fmaf(b, *p, x);
-            }
-        }
-    }
-}
 
 __global__ void __launch_bounds__(K1_MAX_THREADS, 1)
 compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__ items, const __grid_constant__ SeedTable seeds,
@@ -138,7 +107,9 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
             ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), S);                   // every CTA of the cluster has consumed the stage
         }
         ptx::mbar_init(ptx::smem_addr(&ctl->acc_full), 1);
+        for (int k = 0; k < 16; ++k) ptx::mbar_init(ptx::smem_addr(&ctl->old_full[k]), 1);
         ctl->abort = 0;
+        for (int k = 0; k < 4; ++k) ctl->epi_go[k] = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
     }
@@ -275,44 +246,102 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->slice_ready[s]));
             }
         }
-        if (warp < 6 && ok && item.tiles > 0) {
-            // epilogue: warp w reads tensor-memory lanes 32*(w%4) .. +31, i.e. rows of the tile
+        // Epilogue.  The generator warps, now idle, form groups of four; warp w of a group owns tensor-memory lanes
+        // 32*(w%4) .. +31, i.e. those rows of every tile.  The accumulators leave in chunks of 32 columns x 128 rows
+        // (16 KB), dealt round-robin to the groups: registers -> shared memory in the 128-byte-swizzled layout of the
+        // sketch's tensor map -> one bulk tensor operation per chunk, which the hardware clips at the sketch's last row
+        // and column:
+        //   add   S <- S + a*acc   (b == 1, or several items share the rows and S was scaled by b beforehand):
+        //         a bulk reduction, nothing is read back;
+        //   store S <- a*acc       (b == 0 and the item owns its rows);
+        //   rmw   S <- b*S + a*acc (the item owns its rows): the old chunk comes in by a bulk load, one chunk ahead.
+        // The chunk buffers are the tiles of the ring, which nothing uses once the last MMA has completed.
+        const int gw = warp - 2;
+        const int slots_per_stage = T + (int)(a_bytes / (uint32_t)G_TILE_BYTES);   // 16 KB areas of one stage
+        const int areas = stages * slots_per_stage;
+        const int EG = min(min(GW >> 2, 4), areas);               // groups at work
+        if (gw < 4 * EG && item.tiles > 0) {
+            const int grp = gw >> 2;
+            const bool leader = (gw & 3) == 0 && lane == 0;
             const int quarter = warp & 3;
-            if (ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full), 0, abort)) {
-                ptx::tc_fence_after_sync();
-                if (late_wait) ptx::grid_dependency_wait();
-                const bool vec_ok = ((mat->lds & 3) == 0) && ((reinterpret_cast<uintptr_t>(mat->S) & 15) == 0);
-                // S <- S + a*acc needs no read; a split item adds into rows that were scaled by b beforehand
-                const bool add_only = item.direct == 0 || b == 1.0f;
-                for (int t = 0; t < item.tiles; ++t) {
-                    const int64_t row = (int64_t)item.row0 + t * 128 + quarter * 32 + lane;
-                    const bool live = row < mat->n;
-                    float* srow = mat->S + row * mat->lds;
-                    // the owner of a row reads its old values 32 columns at a time before the accumulator is fetched,
-                    // so the eight loads are in flight together
-                    const bool rmw = live && !add_only && b != 0.0f && vec_ok;
-                    for (int j32 = 0; j32 < r_pad; j32 += 32) {
-                        float4 old[2][4] = {};
+            const int trow = quarter * 32 + lane;                 // row inside a tile
+            const uint32_t bar_a = 1u + 2u * (uint32_t)grp, bar_b = bar_a + 1u;
+            const bool acc_ok = ok && ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full), 0, abort);
+            ptx::tc_fence_after_sync();
+            if (late_wait) ptx::grid_dependency_wait();
+            const bool add = item.direct == 0 || b == 1.0f;
+            const bool rmw = !add && b != 0.0f;
+            const int nchunks = (r + 31) >> 5;
+            const int total = item.tiles * nchunks;               // chunks of this CTA; the group takes grp, grp + EG, ...
+            const int NB = min(areas / EG, 4);                    // buffers of this group
+            auto buffer = [&](int u) {                            // u: running index of the group's chunks
+                const int k = grp * NB + u % NB;
+                return smem_base + (uint32_t)(k / slots_per_stage) * stage_bytes + (uint32_t)(k % slots_per_stage) * G_TILE_BYTES;
+            };
+            auto wait_reads = [&]() {                             // all but the newest NB-2 stores have been read out of shared memory
+                if (NB >= 4) ptx::tma_store_wait_read<2>();
+                else if (NB == 3) ptx::tma_store_wait_read<1>();
+                else ptx::tma_store_wait_read<0>();
+            };
+            auto load_old = [&](int u) {
+                const int i = grp + u * EG;
+                const uint32_t bar = ptx::smem_addr(&ctl->old_full[grp * 4 + u % NB]);
+                ptx::mbar_arrive_expect_tx(bar, S_CHUNK_BYTES_K1);
+                ptx::tma_load_2d(buffer(u), &mat->map_s, (i % nchunks) * 32, item.row0 + (i / nchunks) * 128, bar);
+            };
+            const int mine = (total - grp + EG - 1) / EG;
+            for (int u = 0; u < mine; ++u) {
+                const int i = grp + u * EG;
+                if (leader) {
+                    const bool go = acc_ok && !*abort;
+                    if (go) {
+                        wait_reads();
                         if (rmw) {
-#pragma unroll
-                            for (int q = 0; q < 2; ++q)
-#pragma unroll
-                                for (int u = 0; u < 4; ++u)
-                                    if (j32 + 16 * q + 4 * u + 4 <= r) old[q][u] = *reinterpret_cast<const float4*>(srow + j32 + 16 * q + 4 * u);
-                        }
-#pragma unroll
-                        for (int q = 0; q < 2; ++q) {
-                            const int j0 = j32 + 16 * q;
-                            if (j0 < r_pad) {
-                                uint32_t v[16];
-                                ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + t * r_pad + j0, v);
-                                ptx::tmem_ld_wait();
-                                if (live) k1_store_chunk(srow, v, old[q], j0, r, a, b, add_only, vec_ok);
-                            }
+                            if (u == 0) load_old(0);
+                            if (NB > 1 && u + 1 < mine) load_old(u + 1);
+                            else if (NB == 1 && u > 0) load_old(u);
                         }
                     }
+                    ctl->epi_go[grp] = go ? 1 : 0;
+                }
+                ptx::named_barrier_sync(bar_a, 128);
+                if (!*(volatile int*)&ctl->epi_go[grp]) break;    // uniform: written before the barrier by one thread
+                const int t = i / nchunks, c = i % nchunks;
+                uint32_t v[32];
+                ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + t * r_pad + c * 32, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                if (c * 32 + 16 < r_pad)
+                    ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + t * r_pad + c * 32 + 16, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+                else {
+#pragma unroll
+                    for (int k = 16; k < 32; ++k) v[k] = 0u;
+                }
+                ptx::tmem_ld_wait();
+                const uint32_t brow = buffer(u) + (uint32_t)trow * 128u;
+                if (rmw) ptx::mbar_wait(ptx::smem_addr(&ctl->old_full[grp * 4 + u % NB]), (uint32_t)(u / NB) & 1u, abort);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const uint32_t addr = brow + (uint32_t)((q ^ (trow & 7)) << 4);
+                    float x0 = a * __uint_as_float(v[4 * q]), x1 = a * __uint_as_float(v[4 * q + 1]);
+                    float x2 = a * __uint_as_float(v[4 * q + 2]), x3 = a * __uint_as_float(v[4 * q + 3]);
+                    if (rmw) {
+                        uint32_t o0, o1, o2, o3;
+                        ptx::ld_shared_v4(addr, o0, o1, o2, o3);
+                        x0 = fmaf(b, __uint_as_float(o0), x0);
+                        x1 = fmaf(b, __uint_as_float(o1), x1);
+                        x2 = fmaf(b, __uint_as_float(o2), x2);
+                        x3 = fmaf(b, __uint_as_float(o3), x3);
+                    }
+                    ptx::st_shared_v4(addr, __float_as_uint(x0), __float_as_uint(x1), __float_as_uint(x2), __float_as_uint(x3));
+                }
+                ptx::fence_proxy_async_smem();
+                ptx::named_barrier_sync(bar_b, 128);
+                if (leader && !*abort) {
+                    if (add) ptx::tma_reduce_add_2d(&mat->map_s, c * 32, item.row0 + t * 128, buffer(u));
+                    else ptx::tma_store_2d(&mat->map_s, c * 32, item.row0 + t * 128, buffer(u));
+                    ptx::tma_store_commit();
                 }
             }
+            if (leader) ptx::tma_store_wait_all<0>();             // the sketch is complete in global memory before the CTA ends
         }
     }
     ptx::tc_fence_before_sync();
@@ -1127,7 +1156,8 @@ inline flora_status tc_fill_matrices(TcSet& set, const std::vector<flora_mat>& G
         tm.n = (int32_t)big.rows;
         tm.m = (int32_t)big.cols;
         if (!G.empty() && G[i].rows && G[i].cols && !make_map(&tm.map_g, G[i])) return FLORA_ERR_CUDA;
-        if (!W.empty() && W[i].rows && W[i].cols && (!make_map(&tm.map_w, W[i]) || !make_map_f32(&tm.map_s, S[i]))) return FLORA_ERR_CUDA;
+        if (!W.empty() && W[i].rows && W[i].cols && !make_map(&tm.map_w, W[i])) return FLORA_ERR_CUDA;
+        if (S[i].rows && S[i].cols && !make_map_f32(&tm.map_s, S[i])) return FLORA_ERR_CUDA;
     }
     return FLORA_OK;
 }
