@@ -83,7 +83,7 @@ struct K1Smem {                            // barriers and scalars, placed after
 
 __global__ void __launch_bounds__(K1_MAX_THREADS, 1)
 compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__ items, const __grid_constant__ SeedTable seeds,
-                   int seed_base, int r, float scale, float a, float b, int T, int stages, int S, int GW, int late_wait)
+                   int seed_base, int r, float scale, float a, float b, int T, int stages, int S, int GW, int P, int late_wait)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
@@ -102,8 +102,8 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->full_g[s]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctl->full_a[s]), S > 1 ? 1 : GW);   // cluster: one arrival + the peers' bytes
-            ptx::mbar_init(ptx::smem_addr(&ctl->slice_ready[s]), GW);
+            ptx::mbar_init(ptx::smem_addr(&ctl->full_a[s]), S > 1 ? 1 : GW / P);   // cluster: one arrival + the peers' bytes
+            ptx::mbar_init(ptx::smem_addr(&ctl->slice_ready[s]), GW / P);
             ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), S);                   // every CTA of the cluster has consumed the stage
         }
         ptx::mbar_init(ptx::smem_addr(&ctl->acc_full), 1);
@@ -207,11 +207,16 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
         }
     } else {
         // ------------------------------------------------------------------ generators, then epilogue
-        const int g = threadIdx.x - 64;                       // 0 .. 32*GW-1
+        // The generator warps form P teams; team p writes the tiles of the steps p, p + P, ...: a thread's task (eight
+        // values) is a long dependent chain, so with few tasks per thread it is latency, not issue rate, that bounds one
+        // tile, and teams working on neighbouring steps at the same time hide it.
+        const int team_threads = 32 * (GW / P);
+        const int team = (threadIdx.x - 64) / team_threads;
+        const int g = (threadIdx.x - 64) - team * team_threads;   // 0 .. team_threads-1
         const PhiloxKey key = make_key(seeds.s[item.mat - seed_base]);
         const int tasks = r * 8;                              // (row j, 16-byte chunk c) pairs of one A tile
         bool ok = true;
-        for (int ks = 0; ks < item.ksteps && ok; ++ks) {
+        for (int ks = team; ks < item.ksteps && ok; ks += P) {
             const int s = ks % stages, it = ks / stages;
             ok = S > 1 ? ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort)
                        : ptx::mbar_wait(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort);
@@ -219,7 +224,7 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
             const uint32_t a_tile = smem_base + s * stage_bytes + T * G_TILE_BYTES;
             const uint32_t q0 = (uint32_t)(item.kstep0 + ks) * 16u;
             if (S == 1) {
-                for (int t = g; t < tasks; t += 32 * GW) {
+                for (int t = g; t < tasks; t += team_threads) {
                     const int j = t >> 3, c = t & 7;
                     const uint2 lo = projection_quad_bf16(q0 + 2 * c, (uint32_t)j, key, scale);
                     const uint2 hi = projection_quad_bf16(q0 + 2 * c + 1, (uint32_t)j, key, scale);
@@ -233,7 +238,7 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
                 // [rank, rank+1) * r_pad/S of the tile in its own shared memory; the forwarder warp sends them on
                 const int rows_per_cta = r_pad / S;
                 const int my_tasks = rows_per_cta * 8;
-                for (int t = g; t < my_tasks; t += 32 * GW) {
+                for (int t = g; t < my_tasks; t += team_threads) {
                     const int j = (int)rank * rows_per_cta + (t >> 3), c = t & 7;
                     if (j < r) {
                         const uint2 lo = projection_quad_bf16(q0 + 2 * c, (uint32_t)j, key, scale);
@@ -713,7 +718,7 @@ struct TcSet {
     bool decompress_ready = false;
     bool transient = false;             // device buffers come from the stream-ordered allocator
     int count = 0, r = 0;
-    int T = 1, stages = 2, S = 1, GW = 8;
+    int T = 1, stages = 2, S = 1, GW = 8, P = 1;
     std::vector<int> k1_launch_first_mat;
     size_t k1_smem = 0;
     TcMatrix* d_mats = nullptr;
@@ -873,6 +878,15 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
     int GW = (per_sm == 1 && ratio / S > 0.15) ? 16 : 8;
     GW = tune_knob("FLORA_K1_GEN_WARPS", GW, 4, per_sm == 1 ? K1_MAX_GEN_WARPS : 8);
     set.GW = GW;
+    // generator teams: as many as keep every thread of a team busy with at least one task per tile
+    {
+        const int tile_tasks = (S > 1 ? r_pad / S : r) * 8;
+        int P = 1;
+        while (2 * P <= stages && GW % (2 * P) == 0 && 32 * GW / (2 * P) >= tile_tasks) P *= 2;
+        P = tune_knob("FLORA_K1_TEAMS", P, 1, 8);
+        while (P > 1 && (GW % P || P > stages || (P & (P - 1)))) --P;
+        set.P = P;
+    }
     set.T = T;
     set.S = S;
     set.stages = stages;
@@ -1299,7 +1313,7 @@ inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, 
         cfg.numAttrs = set.S > 1 ? 2 : 1;
         const TcMatrix* mats = set.d_mats;
         const K1Item* items = set.d_k1 + begin;
-        if (cudaLaunchKernelEx(&cfg, compress_tc_kernel, mats, items, table, seed_base, r, scale, a, b, set.T, set.stages, set.S, set.GW, l == 0 ? late_wait : 0) !=
+        if (cudaLaunchKernelEx(&cfg, compress_tc_kernel, mats, items, table, seed_base, r, scale, a, b, set.T, set.stages, set.S, set.GW, set.P, l == 0 ? late_wait : 0) !=
             cudaSuccess)
             return FLORA_ERR_CUDA;
         launches.fetch_add(1, std::memory_order_relaxed);
