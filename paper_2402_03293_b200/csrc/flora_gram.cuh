@@ -33,7 +33,7 @@ struct GramJob {            // one matrix
 
 struct GramItem {           // one CTA of the gram kernel
     int32_t job;
-    int32_t kstep0;         // first 64-column step
+    int32_t kstep0;         // first step (a step is kw = 16, 32 or 64 columns, the same for the whole launch)
     int32_t ksteps;
     int32_t pad;
 };
@@ -59,7 +59,7 @@ __device__ __forceinline__ uint32_t mask_pair(uint32_t w, int64_t col, int64_t m
 template <bool SINGLE>
 __global__ void __launch_bounds__(GRAM_THREADS, 1)
 gram_tc_kernel(const GramJob* __restrict__ jobs, const GramItem* __restrict__ items, const __grid_constant__ GramJob single, int per_steps,
-               int r, float scale)
+               int r, float scale, int kw)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
@@ -72,7 +72,7 @@ gram_tc_kernel(const GramJob* __restrict__ jobs, const GramItem* __restrict__ it
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     GramItem item;
     if (SINGLE) {
-        const int total = (single.m + 63) >> 6;
+        const int total = (single.m + kw - 1) / kw;
         item.job = 0;
         item.kstep0 = (int)blockIdx.x * per_steps;
         item.ksteps = min(per_steps, total - item.kstep0);
@@ -125,8 +125,7 @@ gram_tc_kernel(const GramJob* __restrict__ jobs, const GramItem* __restrict__ it
                 const uint64_t d_old = desc_base + (uint64_t)((s * stage_bytes) >> 4);
                 const uint64_t d_new = d_old + (uint64_t)(old_bytes >> 4);
                 for (int h = 0; h < halves; ++h)
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
+                    for (int kk = 0; kk < (kw >> 4); ++kk)
                         ptx::umma_bf16(tmem + h * r_n, d_old + (uint64_t)((h * 128 * 128 + kk * 32) >> 4), d_new + (uint64_t)(kk * 2), idesc,
                                        (ks | kk) != 0);
                 ptx::umma_commit(ptx::smem_addr(&ctl->empty[s]));
@@ -136,20 +135,21 @@ gram_tc_kernel(const GramJob* __restrict__ jobs, const GramItem* __restrict__ it
     } else {
         const int g = threadIdx.x - 32;
         const PhiloxKey key_old = make_key(job.seed_old), key_new = make_key(job.seed_new);
-        const int per_mat = r * 8;                        // (row, 16-byte chunk) tasks of one tile
+        const int cpr = kw >> 3;                          // 16-byte chunks (8 columns) per row of a step: 2, 4 or 8
+        const int per_mat = r * cpr;                      // (row, 16-byte chunk) tasks of one tile
         bool ok = true;
         for (int ks = 0; ks < item.ksteps && ok; ++ks) {
             const int s = ks & 1;
             ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty[s]), ((ks >> 1) & 1) ^ 1, abort);
             if (!ok) break;
             const uint32_t st = smem_base + s * stage_bytes;
-            const uint32_t q0 = (uint32_t)(item.kstep0 + ks) * 16u;
-            const int64_t col_base = (int64_t)(item.kstep0 + ks) * 64;
-            const bool ragged = col_base + 64 > job.m;
+            const uint32_t q0 = (uint32_t)(item.kstep0 + ks) * (uint32_t)(kw >> 2);
+            const int64_t col_base = (int64_t)(item.kstep0 + ks) * kw;
+            const bool ragged = col_base + kw > job.m;
             for (int t = g; t < 2 * per_mat; t += 32 * GRAM_GEN_WARPS) {
                 const bool is_new = t >= per_mat;
                 const int tt = is_new ? t - per_mat : t;
-                const int j = tt >> 3, c = tt & 7;
+                const int j = tt / cpr, c = tt % cpr;
                 const PhiloxKey key = is_new ? key_new : key_old;
                 uint2 lo = projection_quad_bf16(q0 + 2 * c, (uint32_t)j, key, scale);
                 uint2 hi = projection_quad_bf16(q0 + 2 * c + 1, (uint32_t)j, key, scale);
@@ -204,13 +204,14 @@ gram_tc_kernel(const GramJob* __restrict__ jobs, const GramItem* __restrict__ it
     }
 }
 
+// Fallback of the kernel below for sketches whose rows are not 16-byte aligned or whose rank is no multiple of 4.
 // dst[i,:] <- bb dst[i,:] + aa src[i,:] T for every job (or the one passed by value); blockIdx.y = job.  A block
 // takes 8 rows and has one thread per column of the sketch (r rounded up to whole warps); the rows are staged in
 // shared memory first, so dst may alias src.
 constexpr int APPLY_ROWS = 8;
 template <bool SINGLE>
 __global__ void __launch_bounds__(256)
-apply_gram_jobs_kernel(const GramJob* __restrict__ jobs, const __grid_constant__ GramJob single, int r, float aa, float bb)
+apply_gram_rows_kernel(const GramJob* __restrict__ jobs, const __grid_constant__ GramJob single, int r, float aa, float bb)
 {
     __shared__ float Ss[APPLY_ROWS][256];
     const GramJob job = SINGLE ? single : jobs[blockIdx.y];
@@ -240,6 +241,98 @@ apply_gram_jobs_kernel(const GramJob* __restrict__ jobs, const __grid_constant__
     }
 }
 
+// dst[i,:] <- bb dst[i,:] + aa src[i,:] T for every job (or the one passed by value); blockIdx.y = job.
+// Register-tiled: a thread owns 8 rows x 4 columns of the output; per four steps of the inner index it reads four
+// 16-byte pieces of T and eight of src from shared memory for 128 multiply-adds.  T streams through shared memory in
+// tiles of 16 rows, double-buffered with asynchronous copies; the block's rows of src are staged first, so dst may
+// alias src.  Needs r % 4 == 0 and 16-byte aligned rows of src, dst and T.
+constexpr int APPLY_RT = 8;                 // rows per thread
+constexpr int APPLY_AC = 16;                // rows of T per tile
+constexpr int APPLY_SRC_FLOATS = 9728;      // >= rows_per_block * (r + 4) for every r <= 256
+inline int apply_row_groups(int r) { return std::min(256 / (r >> 2), 32); }
+inline size_t apply_smem_bytes(int r) { return sizeof(float) * ((size_t)APPLY_SRC_FLOATS + 2 * (size_t)APPLY_AC * r); }
+template <bool SINGLE>
+__global__ void __launch_bounds__(256)
+apply_gram_jobs_kernel(const GramJob* __restrict__ jobs, const __grid_constant__ GramJob single, int r, int row_groups, float aa, float bb)
+{
+    extern __shared__ __align__(16) float apply_smem[];
+    float* Ss = apply_smem;
+    float* Ts = apply_smem + APPLY_SRC_FLOATS;                 // two tiles of APPLY_AC x r
+    const GramJob job = SINGLE ? single : jobs[blockIdx.y];
+    const int tid = threadIdx.x;
+    const int cgs = r >> 2, rs = r + 4;                        // column groups; padded row stride of the src rows
+    const int rows = row_groups * APPLY_RT;
+    const int64_t row0 = (int64_t)blockIdx.x * rows;
+    if (row0 >= job.n) return;
+    const int ntiles = (r + APPLY_AC - 1) / APPLY_AC;
+    auto load_tile = [&](int k) {
+        const int a0 = k * APPLY_AC, na = min(APPLY_AC, r - a0);
+        float* dst = Ts + (k & 1) * APPLY_AC * r;
+        for (int t = tid; t < na * cgs; t += 256) ptx::cp_async_16(ptx::smem_addr(dst + 4 * t), job.T + (int64_t)a0 * r + 4 * t);
+        ptx::cp_async_commit();
+    };
+    load_tile(0);
+    for (int t = tid; t < rows * cgs; t += 256) {
+        const int i = t / cgs, c = t % cgs;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row0 + i < job.n) v = *reinterpret_cast<const float4*>(job.src + (row0 + i) * job.lds + 4 * c);
+        *reinterpret_cast<float4*>(&Ss[i * rs + 4 * c]) = v;
+    }
+    const int rg = tid / cgs, cg = tid % cgs;
+    const bool active = rg < row_groups;
+    float acc[APPLY_RT][4];
+#pragma unroll
+    for (int i = 0; i < APPLY_RT; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+    const float* srow = &Ss[rg * rs];                          // the thread's rows are rg, rg + row_groups, ...: neighbours in a warp hit different banks
+    for (int k = 0; k < ntiles; ++k) {
+        if (k + 1 < ntiles) {
+            load_tile(k + 1);
+            ptx::cp_async_wait<1>();
+        } else {
+            ptx::cp_async_wait<0>();
+        }
+        __syncthreads();                                       // tile k (and, the first time, the src rows) visible to all
+        if (active) {
+            const int a0 = k * APPLY_AC, na = min(APPLY_AC, r - a0);
+            const float* tt = Ts + (k & 1) * APPLY_AC * r + 4 * cg;
+            for (int al = 0; al < na; al += 4) {
+                float4 t[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) t[u] = *reinterpret_cast<const float4*>(tt + (al + u) * r);
+#pragma unroll
+                for (int i = 0; i < APPLY_RT; ++i) {
+                    const float4 sv = *reinterpret_cast<const float4*>(&srow[i * row_groups * rs + a0 + al]);
+                    const float sa[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {              // same order of accumulation as one thread per column: a ascending
+                        acc[i][0] = fmaf(sa[u], t[u].x, acc[i][0]);
+                        acc[i][1] = fmaf(sa[u], t[u].y, acc[i][1]);
+                        acc[i][2] = fmaf(sa[u], t[u].z, acc[i][2]);
+                        acc[i][3] = fmaf(sa[u], t[u].w, acc[i][3]);
+                    }
+                }
+            }
+        }
+        __syncthreads();                                       // everyone is done with tile k before it is overwritten
+    }
+    if (!active) return;
+#pragma unroll
+    for (int i = 0; i < APPLY_RT; ++i) {
+        const int64_t row = row0 + i * row_groups + rg;
+        if (row < job.n) {
+            float4* p = reinterpret_cast<float4*>(job.dst + row * job.ldd + 4 * cg);
+            float4 o = make_float4(aa * acc[i][0], aa * acc[i][1], aa * acc[i][2], aa * acc[i][3]);
+            if (bb != 0.0f) {
+                const float4 d = *p;
+                o = make_float4(fmaf(bb, d.x, o.x), fmaf(bb, d.y, o.y), fmaf(bb, d.z, o.z), fmaf(bb, d.w, o.w));
+            }
+            *p = o;
+        }
+    }
+}
+
 // Host side.  A set: scratch (r x r per job, job and item tables) from the stream-ordered allocator, a memset, one
 // table upload, the two kernels, the release of the scratch.  A single matrix: only the r x r scratch; the job
 // travels as a kernel parameter.  `jobs` come without T; it is assigned here.
@@ -249,30 +342,43 @@ inline flora_status transfer_tc(std::vector<GramJob>& jobs, int r, float a, floa
     int sms = 148, dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    int64_t total_steps = 0;
+    // step width: 64 columns, or narrower while that leaves fewer than four steps per SM to balance
+    int64_t total_cols = 0;
     int max_n = 1;
     for (const auto& j : jobs) {
-        total_steps += (j.m + 63) / 64;
+        total_cols += j.m;
         max_n = std::max(max_n, j.n);
     }
-    const int64_t chunk = std::max<int64_t>(1, (total_steps + sms - 1) / sms);
+    int kw = 64;
+    while (kw > 16 && total_cols / kw < 4 * (int64_t)sms) kw >>= 1;
+    int64_t total_steps = 0;
+    for (const auto& j : jobs) total_steps += (j.m + kw - 1) / kw;
+    const bool single = jobs.size() == 1;
+    // a single matrix: one wave of equal chunks; a set: about three items per SM, the largest first
+    const int64_t chunk = std::max<int64_t>(1, single ? (total_steps + sms - 1) / sms : (total_steps + 3 * sms - 1) / (3 * sms));
     const size_t t_bytes = (((size_t)r * r * sizeof(float)) + 255) & ~(size_t)255;
     const int r_m = (r + 127) & ~127, r_n = (r + 15) & ~15;
     const size_t smem = 2 * (size_t)(r_m + r_n) * 128 + sizeof(GramSmem) + 1024;
     const float scale = 1.0f / sqrtf((float)r);
-    const bool single = jobs.size() == 1;
-    const unsigned apply_threads = (unsigned)((r + 31) & ~31);        // one thread per sketch column
+    const unsigned apply_threads = (unsigned)((r + 31) & ~31);        // fallback kernel: one thread per sketch column
+    bool tiled = (r & 3) == 0;                                        // register-tiled kernel: 16-byte aligned rows everywhere
+    for (const auto& j : jobs)
+        tiled = tiled && (j.ldd & 3) == 0 && (j.lds & 3) == 0 && (reinterpret_cast<uintptr_t>(j.dst) & 15) == 0 &&
+                (reinterpret_cast<uintptr_t>(j.src) & 15) == 0;
+    const int row_groups = tiled ? apply_row_groups(r) : 0;
+    const unsigned apply_rows = tiled ? (unsigned)(row_groups * APPLY_RT) : (unsigned)APPLY_ROWS;
     std::vector<uint8_t> tables;                 // set: the job table followed by the item table, one upload
     size_t n_items = 0;
     const size_t jobs_bytes = (jobs.size() * sizeof(GramJob) + 255) & ~(size_t)255;
     if (!single) {
         std::vector<GramItem> items;
         for (size_t i = 0; i < jobs.size(); ++i) {
-            const int64_t ks = (jobs[i].m + 63) / 64;
+            const int64_t ks = (jobs[i].m + kw - 1) / kw;
             const int64_t nchunks = std::max<int64_t>(1, (ks + chunk - 1) / chunk);
             const int64_t per = (ks + nchunks - 1) / nchunks;
             for (int64_t k0 = 0; k0 < ks; k0 += per) items.push_back({(int)i, (int)k0, (int)std::min(per, ks - k0), 0});
         }
+        std::stable_sort(items.begin(), items.end(), [](const GramItem& x, const GramItem& y) { return x.ksteps > y.ksteps; });
         n_items = items.size();
         tables.resize(jobs_bytes + items.size() * sizeof(GramItem));
         memcpy(tables.data() + jobs_bytes, items.data(), items.size() * sizeof(GramItem));
@@ -286,15 +392,21 @@ inline flora_status transfer_tc(std::vector<GramJob>& jobs, int r, float a, floa
     for (size_t i = 0; i < jobs.size(); ++i) jobs[i].T = reinterpret_cast<float*>(buf + i * t_bytes);
     flora_status rc = FLORA_OK;
     bool ok = cudaMemsetAsync(buf, 0, tables_off, st) == cudaSuccess;
+    if (tiled)
+        ok = ok && (single ? cudaFuncSetAttribute(apply_gram_jobs_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apply_smem_bytes(r))
+                           : cudaFuncSetAttribute(apply_gram_jobs_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apply_smem_bytes(r))) ==
+                       cudaSuccess;
     if (single) {
         ok = ok && cudaFuncSetAttribute(gram_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess;
         if (ok) {
-            const int ks = (jobs[0].m + 63) / 64;
+            const int ks = (jobs[0].m + kw - 1) / kw;
             if (ks > 0) {
-                gram_tc_kernel<true><<<(unsigned)((ks + chunk - 1) / chunk), GRAM_THREADS, smem, st>>>(nullptr, nullptr, jobs[0], (int)chunk, r, scale);
+                gram_tc_kernel<true><<<(unsigned)((ks + chunk - 1) / chunk), GRAM_THREADS, smem, st>>>(nullptr, nullptr, jobs[0], (int)chunk, r, scale, kw);
                 launches.fetch_add(1, std::memory_order_relaxed);
             }
-            apply_gram_jobs_kernel<true><<<dim3((unsigned)((max_n + APPLY_ROWS - 1) / APPLY_ROWS), 1), apply_threads, 0, st>>>(nullptr, jobs[0], r, a, b);
+            const dim3 grid((unsigned)((max_n + apply_rows - 1) / apply_rows), 1);
+            if (tiled) apply_gram_jobs_kernel<true><<<grid, 256, apply_smem_bytes(r), st>>>(nullptr, jobs[0], r, row_groups, a, b);
+            else apply_gram_rows_kernel<true><<<grid, apply_threads, 0, st>>>(nullptr, jobs[0], r, a, b);
             launches.fetch_add(1, std::memory_order_relaxed);
         }
     } else {
@@ -306,12 +418,13 @@ inline flora_status transfer_tc(std::vector<GramJob>& jobs, int r, float a, floa
             const GramJob* d_jobs = reinterpret_cast<const GramJob*>(buf + tables_off);
             const GramItem* d_items = reinterpret_cast<const GramItem*>(buf + tables_off + jobs_bytes);
             if (n_items) {
-                gram_tc_kernel<false><<<(unsigned)n_items, GRAM_THREADS, smem, st>>>(d_jobs, d_items, jobs[0], 0, r, scale);
+                gram_tc_kernel<false><<<(unsigned)n_items, GRAM_THREADS, smem, st>>>(d_jobs, d_items, jobs[0], 0, r, scale, kw);
                 launches.fetch_add(1, std::memory_order_relaxed);
             }
             for (size_t begin = 0; begin < jobs.size(); begin += 65535) {
-                dim3 grid((unsigned)((max_n + APPLY_ROWS - 1) / APPLY_ROWS), (unsigned)std::min<size_t>(65535, jobs.size() - begin));
-                apply_gram_jobs_kernel<false><<<grid, apply_threads, 0, st>>>(d_jobs + begin, jobs[0], r, a, b);
+                dim3 grid((unsigned)((max_n + apply_rows - 1) / apply_rows), (unsigned)std::min<size_t>(65535, jobs.size() - begin));
+                if (tiled) apply_gram_jobs_kernel<false><<<grid, 256, apply_smem_bytes(r), st>>>(d_jobs + begin, jobs[0], r, row_groups, a, b);
+                else apply_gram_rows_kernel<false><<<grid, apply_threads, 0, st>>>(d_jobs + begin, jobs[0], r, a, b);
                 launches.fetch_add(1, std::memory_order_relaxed);
             }
         }
