@@ -93,7 +93,7 @@ def test_decompress_apply(n, m, r, dtype, force_simt):
 
 @pytest.mark.parametrize("operand", ["f32", "bf16"])
 @pytest.mark.parametrize("n,m,r", [(1, 1, 1), (9, 33, 4), (100, 515, 32), (257, 1024, 64), (40, 300, 256), (300, 11008, 200),
-                                   (64, 4097, 130), (1000, 64, 8), (33, 70, 17)])
+                                   (64, 4097, 130), (1000, 64, 8), (33, 70, 17), (64, 20000, 64), (40, 40010, 16)])
 def test_transfer(n, m, r, operand):
     M0 = torch.randn(n, r, device=DEV)
     M = M0.clone()
