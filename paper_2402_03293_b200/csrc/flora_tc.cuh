@@ -814,7 +814,7 @@ inline int sm_count()
     return n;
 }
 
-constexpr size_t SMEM_BUDGET = 224 * 1024;   // per SM, below the 227 KB limit of sm_100
+constexpr size_t SMEM_BUDGET = 226 * 1024;   // per SM, below the 227 KB limit of sm_100
 
 // Tuning knobs (environment variables, read when a set is planned): they change tile shapes and the
 // work split only, never what is computed.
@@ -1027,9 +1027,12 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
     const bool bf16s = tune_knob("FLORA_K2_BF16S", r > 64 ? 1 : 0, 0, 1) != 0;
     set.k2_bf16 = bf16s;
     const int kchunks = bf16s ? (r + 63) / 64 : (r + 31) / 32;
-    int bn = kchunks > 2 ? 64 : 128;
+    // slabs of 128 columns (every chunk of S then serves twice the columns of W) whenever two slabs, two W slots and
+    // two S chunks of that width fit; 64 columns otherwise
+    const size_t ctl = sizeof(K2Smem) + 1024;
+    int bn = (2 * (size_t)kchunks * 128 * 128 + 2 * S_CHUNK_BYTES + 2 * 2 * (size_t)W_BOX_BYTES + ctl <= SMEM_BUDGET) ? 128 : 64;
     bn = tune_knob("FLORA_K2_BN", bn, 64, 128) >= 128 ? 128 : 64;
-    const size_t slab_bytes = (size_t)kchunks * bn * 128, slot = (size_t)(bn / 64) * W_BOX_BYTES, ctl = sizeof(K2Smem) + 1024;
+    const size_t slab_bytes = (size_t)kchunks * bn * 128, slot = (size_t)(bn / 64) * W_BOX_BYTES;
     // two CTAs per SM when two of them fit (each with two slabs, two W slots and one S chunk)
     const size_t per_cta_max = 113 * 1024;                       // half of an SM's shared memory minus the reserve
     int per_sm = (2 * slab_bytes + S_CHUNK_BYTES + 2 * slot + ctl <= per_cta_max) ? 2 : 1;
