@@ -1,6 +1,7 @@
 // C ABI of the Flora hot path (see include/flora.h for the contract of every entry point).
 // This file validates arguments, picks a kernel family and launches; all arithmetic of the path
-// lives in the kernels of flora_simt.cuh (fp32 SIMT) and flora_tc.cuh (tcgen05 tensor cores).
+// lives in the kernels of flora_simt.cuh (fp32 SIMT), flora_tc.cuh (tcgen05 tensor cores; host side in flora_tc_host.cuh)
+// and flora_gram.cuh (momentum transfer).
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
@@ -15,7 +16,7 @@
 #include "../../include/flora.h"
 #include "flora_rng.cuh"
 #include "flora_simt.cuh"
-#include "flora_tc.cuh"
+#include "flora_tc_host.cuh"
 #include "flora_gram.cuh"
 
 using namespace flora;
