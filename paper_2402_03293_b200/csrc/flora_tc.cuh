@@ -372,6 +372,7 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
 // ------------------------------------------------------------------------------------------------
 constexpr int K2_FIXED_WARPS = 12;  // warp 0: W loads, 1: MMA, 2-5 and 8-11: combine, 6: S loads, 7: W stores, 12..: slab generators
 constexpr int K2_MAX_GEN_WARPS = 8;
+constexpr int K2_HELPER_WARPS = 8;    // the combine warps, idle until the first tile arrives, generate part of the CTA's first slab
 constexpr int K2_MAX_THREADS = 32 * (K2_FIXED_WARPS + K2_MAX_GEN_WARPS);
 constexpr int K2_MAX_SLOTS = 6;
 constexpr int K2_MAX_CSTAGES = 8;
@@ -380,10 +381,60 @@ constexpr int S_CHUNK_BYTES = 128 * 128;   // 128 rows x 32 fp32
 
 struct K2Smem {
     uint64_t w_full[K2_MAX_SLOTS], w_free[K2_MAX_SLOTS], out_ready[K2_MAX_SLOTS];
-    uint64_t c_full[K2_MAX_CSTAGES], c_empty[K2_MAX_CSTAGES], acc_full[2], acc_empty[2], slab_full[2], slab_empty[2];
+    uint64_t c_full[K2_MAX_CSTAGES], c_empty[K2_MAX_CSTAGES], acc_full[2], acc_empty[2], slab_full[2], slab_empty[2], slab0_help;
     uint32_t tmem_base;
     int abort;
 };
+
+// Writes the tasks first, first + stride, ... of one r x bn slab of A as the N x K operand: row = column of W,
+// K = index j of the sketch, values rounded to bf16 (kept in 32-bit containers, exact in tf32, for the fp32 sketch
+// path).  One task makes a 4-column x 4-j (or 8-j) block and stores one 16-byte chunk per column; j >= r is zero.
+template <bool BF16S>
+__device__ __forceinline__ void k2_generate_slab(uint32_t slab, uint32_t slab_block, int kchunks, int bn, int col0, int r, const PhiloxKey key,
+                                                 float scale, int first, int stride)
+{
+    const int jgroups = kchunks * 8;
+    const int tasks = (bn >> 2) * jgroups;
+    for (int t = first; t < tasks; t += stride) {
+        const int jg = t % jgroups, cq = t / jgroups;       // jg: 16-byte chunk along K (4 tf32 or 8 bf16 values)
+        const uint32_t blk = slab + (jg >> 3) * slab_block;
+        if (BF16S) {
+            uint32_t packed[4][4];
+#pragma unroll
+            for (int jj = 0; jj < 8; jj += 2) {
+                float v0[4] = {0.f, 0.f, 0.f, 0.f}, v1[4] = {0.f, 0.f, 0.f, 0.f};
+                const int j = jg * 8 + jj;
+                if (j < r) projection_quad((uint32_t)(col0 / 4 + cq), (uint32_t)j, key, scale, v0);
+                if (j + 1 < r) projection_quad((uint32_t)(col0 / 4 + cq), (uint32_t)(j + 1), key, scale, v1);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    __nv_bfloat162 pr = __floats2bfloat162_rn(v0[u], v1[u]);
+                    packed[u][jj >> 1] = *reinterpret_cast<uint32_t*>(&pr);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int c = cq * 4 + u;
+                ptx::st_shared_v4(blk + c * 128 + (((jg & 7) ^ (c & 7)) << 4), packed[u][0], packed[u][1], packed[u][2], packed[u][3]);
+            }
+        } else {
+            float v[4][4];
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                float q[4] = {0.f, 0.f, 0.f, 0.f};
+                if (jg * 4 + jj < r) projection_quad((uint32_t)(col0 / 4 + cq), (uint32_t)(jg * 4 + jj), key, scale, q);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) v[u][jj] = bf16_round(q[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int c = cq * 4 + u;
+                ptx::st_shared_v4(blk + c * 128 + (((jg & 7) ^ (c & 7)) << 4), __float_as_uint(v[u][0]), __float_as_uint(v[u][1]),
+                                  __float_as_uint(v[u][2]), __float_as_uint(v[u][3]));
+            }
+        }
+    }
+}
 
 template <bool BF16S>
 __global__ void __launch_bounds__(K2_MAX_THREADS, 1)
@@ -422,6 +473,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
             ptx::mbar_init(ptx::smem_addr(&ctl->slab_full[s]), GW);
             ptx::mbar_init(ptx::smem_addr(&ctl->slab_empty[s]), 1);
         }
+        ptx::mbar_init(ptx::smem_addr(&ctl->slab0_help), K2_HELPER_WARPS);
         ctl->abort = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
@@ -492,6 +544,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
                 const K2Item item = items[it];
                 const uint64_t desc_slab = ptx::umma_desc_k_sw128(slab0 + (k & 1) * slab_bytes);
                 ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_full[k & 1]), (k >> 1) & 1, abort);
+                if (k == 0 && ok) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab0_help), 0, abort);    // the combine warps' share of the first slab
                 for (int i = 0; i < item.tiles && ok; ++i, ++gt) {
                     const uint32_t acc_addr = tmem + (gt & 1) * bn;
                     ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[gt & 1]), ((gt >> 1) & 1) ^ 1, abort);
@@ -557,6 +610,16 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         const int per_half = boxes << 1;                       // 16-column chunks per half: 2 (bn 64) or 4 (bn 128)
         int gt = 0;
         bool ok = true;
+        if ((int)blockIdx.x < n_items) {
+            // nothing to combine yet: write a share of the CTA's first slab alongside the generator warps
+            const K2Item first = items[blockIdx.x];
+            const int helper = (half * 4 + (warp - (half ? 8 : 2))) * 32 + lane;          // 0 .. 255
+            k2_generate_slab<BF16S>(slab0, slab_block, kchunks, bn, first.col0, r, make_key(seeds.s[first.mat - seed_base]), scale,
+                                    32 * GW + helper, 32 * (GW + K2_HELPER_WARPS));
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->slab0_help));
+        }
         for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
             const K2Item item = items[it];
             const int live_chunks = min(boxes, (mats[item.mat].m - item.col0 + 63) >> 6) << 2;
@@ -611,8 +674,6 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         // and widened to 32 bits (exact in tf32).  One task makes a 4-column x 4-j block (four Philox blocks) and
         // stores one 16-byte chunk per column; j >= r is written as zero.
         const int g = threadIdx.x - 32 * K2_FIXED_WARPS;
-        const int jgroups = kchunks * 8;
-        const int tasks = (bn >> 2) * jgroups;
         int k = 0;
         bool ok = true;
         for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++k) {
@@ -621,45 +682,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
             ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_empty[k & 1]), ((k >> 1) & 1) ^ 1, abort);
             if (!ok) break;
             const uint32_t slab = slab0 + (k & 1) * slab_bytes;
-            for (int t = g; t < tasks; t += 32 * GW) {
-                const int jg = t % jgroups, cq = t / jgroups;       // jg: 16-byte chunk along K (4 tf32 or 8 bf16 values)
-                const uint32_t blk = slab + (jg >> 3) * slab_block;
-                if (BF16S) {
-                    uint32_t packed[4][4];
-#pragma unroll
-                    for (int jj = 0; jj < 8; jj += 2) {
-                        float v0[4] = {0.f, 0.f, 0.f, 0.f}, v1[4] = {0.f, 0.f, 0.f, 0.f};
-                        const int j = jg * 8 + jj;
-                        if (j < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)j, key, scale, v0);
-                        if (j + 1 < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)(j + 1), key, scale, v1);
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            __nv_bfloat162 pr = __floats2bfloat162_rn(v0[u], v1[u]);
-                            packed[u][jj >> 1] = *reinterpret_cast<uint32_t*>(&pr);
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int c = cq * 4 + u;
-                        ptx::st_shared_v4(blk + c * 128 + (((jg & 7) ^ (c & 7)) << 4), packed[u][0], packed[u][1], packed[u][2], packed[u][3]);
-                    }
-                } else {
-                    float v[4][4];
-#pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                        float q[4] = {0.f, 0.f, 0.f, 0.f};
-                        if (jg * 4 + jj < r) projection_quad((uint32_t)(item.col0 / 4 + cq), (uint32_t)(jg * 4 + jj), key, scale, q);
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) v[u][jj] = bf16_round(q[u]);
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int c = cq * 4 + u;
-                        ptx::st_shared_v4(blk + c * 128 + (((jg & 7) ^ (c & 7)) << 4), __float_as_uint(v[u][0]), __float_as_uint(v[u][1]),
-                                          __float_as_uint(v[u][2]), __float_as_uint(v[u][3]));
-                    }
-                }
-            }
+            k2_generate_slab<BF16S>(slab, slab_block, kchunks, bn, item.col0, r, key, scale, g, k == 0 ? 32 * (GW + K2_HELPER_WARPS) : 32 * GW);   // the first slab is shared with the combine warps
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->slab_full[k & 1]));
