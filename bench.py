@@ -251,12 +251,22 @@ def run_flora(args):
     hostG = [[g.cpu().pin_memory() for g in G[k]] for k in range(w.tau)]
     hostW = [torch.empty(n, m, dtype=wl.torch_dtype(w.dtype)).pin_memory() for n, m in w.shapes]
 
+    # the read-back of a step's weights runs on a second stream, so it shares the (full-duplex) link with the next
+    # step's uploads; it must have finished before the next decompression overwrites the weights
+    main, side = torch.cuda.current_stream(), torch.cuda.Stream()
+    updated, read_back = torch.cuda.Event(), torch.cuda.Event()
+    read_back.record(side)
+
     def e2e_step():
         s = seeds()
         for k in range(w.tau):
             sets[k].compress_accumulate_from_host(hostG[k], s)
+        main.wait_event(read_back)
         sets[0].decompress_apply(s, LR, 1.0 / w.tau)
-        sets[0].read_weights_to_host(hostW)
+        updated.record(main)
+        side.wait_event(updated)
+        sets[0].read_weights_to_host(hostW, stream=side)
+        read_back.record(side)
         sets[0].zero_state()
         epoch[0] += 1
 
@@ -265,6 +275,7 @@ def run_flora(args):
     e0.record()
     for _ in range(e2e_steps):
         e2e_step()
+    main.wait_event(read_back)              # the last step's weights have arrived in host memory
     e1.record()
     barrier()
     e2e_agg = replicas.aggregate_throughput(grad_bytes_step, e2e_steps, e0.elapsed_time(e1), dist, dev)
@@ -276,8 +287,12 @@ def run_flora(args):
         from oracle import flora_oracle as orc
         state = {}
         dt, b = oracle_sample_step(w, 12, state)
+        cycles = 1
+        while dt < 10.0 and cycles < 12:                       # about 10 s of oracle work, whole cycles only
+            dt2, b2 = oracle_sample_step(w, 12, state)
+            dt, b, cycles = dt + dt2, b + b2, cycles + 1
         cpu_baseline = {"value": b / dt / 1e9, "unit": "GB/s", "cores": orc.max_threads(), "kind": "oracle",
-                        "sample": f"1 full cycle (tau={w.tau} compress + decompress-apply) over all 48 matrices, {dt:.1f} s wall"}
+                        "sample": f"{cycles} full cycle(s) (tau={w.tau} compress + decompress-apply) over all 48 matrices, {dt:.1f} s wall"}
 
     if rank == 0:
         line = {
