@@ -381,7 +381,7 @@ constexpr int S_CHUNK_BYTES = 128 * 128;   // 128 rows x 32 fp32
 
 struct K2Smem {
     uint64_t w_full[K2_MAX_SLOTS], w_free[K2_MAX_SLOTS], out_ready[K2_MAX_SLOTS];
-    uint64_t c_full[K2_MAX_CSTAGES], c_empty[K2_MAX_CSTAGES], acc_full[2], acc_empty[2], slab_full[2], slab_empty[2], slab0_help;
+    uint64_t c_full[K2_MAX_CSTAGES], c_empty[K2_MAX_CSTAGES], acc_full[2], acc_empty[2], slab_full[2], slab_empty[2], slab_help;
     uint32_t tmem_base;
     int abort;
 };
@@ -440,7 +440,7 @@ template <bool BF16S>
 __global__ void __launch_bounds__(K2_MAX_THREADS, 1)
 decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict__ items, int n_items,
                      const __grid_constant__ SeedTable seeds, int seed_base, int r, float scale, float step, int bn, int slots,
-                     int cstages, int GW)
+                     int cstages, int GW, int nslabs)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
@@ -450,7 +450,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
     const uint32_t slab_block = (uint32_t)bn * 128u;           // one K chunk of a slab
     const uint32_t slab_bytes = kchunks * slab_block;
     const uint32_t slab0 = smem_base;
-    const uint32_t c_ring = slab0 + 2 * slab_bytes;
+    const uint32_t c_ring = slab0 + nslabs * slab_bytes;
     const uint32_t w_ring = c_ring + cstages * (uint32_t)S_CHUNK_BYTES;
     const uint32_t slot_bytes = (uint32_t)boxes * W_BOX_BYTES;
     K2Smem* ctl = reinterpret_cast<K2Smem*>(smem_raw + (w_ring - ptx::smem_addr(smem_raw)) + (size_t)slots * slot_bytes);
@@ -473,7 +473,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
             ptx::mbar_init(ptx::smem_addr(&ctl->slab_full[s]), GW);
             ptx::mbar_init(ptx::smem_addr(&ctl->slab_empty[s]), 1);
         }
-        ptx::mbar_init(ptx::smem_addr(&ctl->slab0_help), K2_HELPER_WARPS);
+        ptx::mbar_init(ptx::smem_addr(&ctl->slab_help), K2_HELPER_WARPS);
         ctl->abort = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
@@ -542,9 +542,11 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
             bool ok = true;
             for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++k) {
                 const K2Item item = items[it];
-                const uint64_t desc_slab = ptx::umma_desc_k_sw128(slab0 + (k & 1) * slab_bytes);
-                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_full[k & 1]), (k >> 1) & 1, abort);
-                if (k == 0 && ok) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab0_help), 0, abort);    // the combine warps' share of the first slab
+                const int sb = k % nslabs, sphase = (k / nslabs) & 1;
+                const uint64_t desc_slab = ptx::umma_desc_k_sw128(slab0 + sb * slab_bytes);
+                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_full[sb]), sphase, abort);
+                // the combine warps' share: of the first slab, or of every slab when there is only one buffer
+                if ((k == 0 || nslabs == 1) && ok) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_help), k & 1, abort);
                 for (int i = 0; i < item.tiles && ok; ++i, ++gt) {
                     const uint32_t acc_addr = tmem + (gt & 1) * bn;
                     ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[gt & 1]), ((gt >> 1) & 1) ^ 1, abort);
@@ -565,7 +567,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
                     }
                     if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->acc_full[gt & 1]));
                 }
-                if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->slab_empty[k & 1]));   // every MMA that reads this slab has completed
+                if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->slab_empty[sb]));   // every MMA that reads this slab has completed
             }
         }
     } else if (warp == 7) {
@@ -610,18 +612,21 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         const int per_half = boxes << 1;                       // 16-column chunks per half: 2 (bn 64) or 4 (bn 128)
         int gt = 0;
         bool ok = true;
-        if ((int)blockIdx.x < n_items) {
-            // nothing to combine yet: write a share of the CTA's first slab alongside the generator warps
-            const K2Item first = items[blockIdx.x];
-            const int helper = (half * 4 + (warp - (half ? 8 : 2))) * 32 + lane;          // 0 .. 255
-            k2_generate_slab<BF16S>(slab0, slab_block, kchunks, bn, first.col0, r, make_key(seeds.s[first.mat - seed_base]), scale,
-                                    32 * GW + helper, 32 * (GW + K2_HELPER_WARPS));
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->slab0_help));
-        }
-        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+        const int helper = (half * 4 + (warp - (half ? 8 : 2))) * 32 + lane;              // 0 .. 255
+        int k = 0;
+        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++k) {
             const K2Item item = items[it];
+            if (k == 0 || nslabs == 1) {
+                // Nothing to combine yet (first item), or a single slab buffer whose refill nothing overlaps: write a
+                // share of the slab alongside the generator warps.
+                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_empty[0]), ((k / nslabs) & 1) ^ 1, abort);
+                if (!ok) break;
+                k2_generate_slab<BF16S>(slab0, slab_block, kchunks, bn, item.col0, r, make_key(seeds.s[item.mat - seed_base]), scale,
+                                        32 * GW + helper, 32 * (GW + K2_HELPER_WARPS));
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->slab_help));
+            }
             const int live_chunks = min(boxes, (mats[item.mat].m - item.col0 + 63) >> 6) << 2;
             const int c_begin = half * per_half;
             const int mine = max(0, min(per_half, live_chunks - c_begin));
@@ -679,13 +684,16 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++k) {
             const K2Item item = items[it];
             const PhiloxKey key = make_key(seeds.s[item.mat - seed_base]);
-            ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_empty[k & 1]), ((k >> 1) & 1) ^ 1, abort);
+            const int sb = k % nslabs;
+            ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_empty[sb]), ((k / nslabs) & 1) ^ 1, abort);
             if (!ok) break;
-            const uint32_t slab = slab0 + (k & 1) * slab_bytes;
-            k2_generate_slab<BF16S>(slab, slab_block, kchunks, bn, item.col0, r, key, scale, g, k == 0 ? 32 * (GW + K2_HELPER_WARPS) : 32 * GW);   // the first slab is shared with the combine warps
+            const uint32_t slab = slab0 + sb * slab_bytes;
+            // the first slab (every slab, with a single buffer) is shared with the combine warps
+            k2_generate_slab<BF16S>(slab, slab_block, kchunks, bn, item.col0, r, key, scale, g,
+                                    (k == 0 || nslabs == 1) ? 32 * (GW + K2_HELPER_WARPS) : 32 * GW);
             ptx::fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->slab_full[k & 1]));
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->slab_full[sb]));
         }
     }
     ptx::tc_fence_before_sync();

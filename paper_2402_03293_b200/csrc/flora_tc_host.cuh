@@ -34,7 +34,7 @@ struct TcSet {
     std::vector<int> k1_launch_begin;   // item ranges per launch (at most SEEDS_PER_LAUNCH matrices each)
     std::vector<int> split_mats;        // matrices whose sketch is updated by several items
     // decompression
-    int bn = 128, slots = 2, cstages = 2, k2_gw = 8, k2_grid_max = 148;
+    int bn = 128, slots = 2, cstages = 2, k2_gw = 8, k2_nslabs = 2, k2_grid_max = 148;
     bool k2_bf16 = false;               // ranks above 64: the kernel reads a bf16 copy of the sketches
     __nv_bfloat16* d_sb = nullptr;      // that copy (scratch owned by the set)
     std::vector<int> k2_launch_first_mat;
@@ -338,8 +338,14 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
     const size_t per_cta_max = 113 * 1024;                       // half of an SM's shared memory minus the reserve
     int per_sm = (2 * slab_bytes + S_CHUNK_BYTES + 2 * slot + ctl <= per_cta_max) ? 2 : 1;
     per_sm = 1;   // twelve fixed warps plus generators: one CTA per SM
-    const size_t budget = (per_sm == 2 ? per_cta_max : SMEM_BUDGET) - ctl - 2 * slab_bytes;
-    int cstages = std::max(2, std::min(kchunks + 1, 4));
+    // Two slab buffers (the next item's slab is generated while the current item streams) unless that leaves fewer
+    // than four S chunks in flight: the chunks of one W tile are kchunks x 16 KB, and with too few of them under way
+    // the loads' latency, not bandwidth, sets the pace.  With one buffer every warp that is idle between two items
+    // (the combine warps) shares the generation.
+    int nslabs = (2 * slab_bytes + 4 * S_CHUNK_BYTES + 2 * slot + ctl <= SMEM_BUDGET) ? 2 : 1;
+    nslabs = tune_knob("FLORA_K2_SLABS", nslabs, 1, 2);
+    const size_t budget = (per_sm == 2 ? per_cta_max : SMEM_BUDGET) - ctl - nslabs * slab_bytes;
+    int cstages = std::max(2, std::min(nslabs == 1 ? 2 * kchunks : kchunks + 1, nslabs == 1 ? K2_MAX_CSTAGES : 4));
     cstages = tune_knob("FLORA_K2_CSTAGES", cstages, 1, K2_MAX_CSTAGES);
     while (cstages > 1 && (size_t)cstages * S_CHUNK_BYTES + 2 * slot > budget) --cstages;
     int slots = (int)std::min<size_t>(K2_MAX_SLOTS, (budget - (size_t)cstages * S_CHUNK_BYTES) / slot);
@@ -350,7 +356,8 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
     set.slots = slots;
     set.cstages = cstages;
     set.k2_gw = GW;
-    set.k2_smem = 2 * slab_bytes + (size_t)cstages * S_CHUNK_BYTES + (size_t)slots * slot + sizeof(K2Smem) + 1024;
+    set.k2_nslabs = nslabs;
+    set.k2_smem = nslabs * slab_bytes + (size_t)cstages * S_CHUNK_BYTES + (size_t)slots * slot + sizeof(K2Smem) + 1024;
     const int grid_max = sm_count() * per_sm;
     // cost model (microseconds of one SM): a tile streams bn*128*4 bytes at the SM's share of HBM; a slab costs
     // r*bn normals at the generator warps' rate and overlaps the previous item's streaming
@@ -388,7 +395,7 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
         for (size_t k = 0; k < sorted.size(); ++k) {
             // generation overlaps the streaming of the previous item, but the two compete for issue slots
             const double stream = sorted[k].tiles * t_tile;
-            t[k % t.size()] += std::max(t_slab, stream) + 0.35 * std::min(t_slab, stream) + 0.2;
+            t[k % t.size()] += nslabs == 1 ? 0.55 * t_slab + stream + 0.2 : std::max(t_slab, stream) + 0.35 * std::min(t_slab, stream) + 0.2;
         }
         return *std::max_element(t.begin(), t.end());
     };
@@ -661,10 +668,10 @@ inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float s
         const int grid = std::min(set.k2_grid_max, end - begin);
         if (set.k2_bf16)
             decompress_tc_kernel<true><<<grid, 32 * (K2_FIXED_WARPS + set.k2_gw), set.k2_smem, st>>>(
-                set.d_mats, set.d_k2 + begin, end - begin, table, seed_base, r, scale, step, set.bn, set.slots, set.cstages, set.k2_gw);
+                set.d_mats, set.d_k2 + begin, end - begin, table, seed_base, r, scale, step, set.bn, set.slots, set.cstages, set.k2_gw, set.k2_nslabs);
         else
             decompress_tc_kernel<false><<<grid, 32 * (K2_FIXED_WARPS + set.k2_gw), set.k2_smem, st>>>(
-                set.d_mats, set.d_k2 + begin, end - begin, table, seed_base, r, scale, step, set.bn, set.slots, set.cstages, set.k2_gw);
+                set.d_mats, set.d_k2 + begin, end - begin, table, seed_base, r, scale, step, set.bn, set.slots, set.cstages, set.k2_gw, set.k2_nslabs);
         launches.fetch_add(1, std::memory_order_relaxed);
     }
     return cudaPeekAtLastError() == cudaSuccess ? FLORA_OK : FLORA_ERR_CUDA;
