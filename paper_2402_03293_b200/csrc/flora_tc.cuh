@@ -75,7 +75,7 @@ constexpr int G_TILE_BYTES = 128 * 128;   // 128 rows x 64 bf16
 constexpr int S_CHUNK_BYTES_K1 = 128 * 128; // 128 rows x 32 fp32
 
 struct K1Smem {                            // barriers and scalars, placed after the tile ring
-    uint64_t full_g[8], full_a[8], slice_ready[8], empty[8], acc_full, old_full[16];
+    uint64_t full_g[8], empty_g[8], full_a[8], slice_ready[8], empty_a[8], acc_full, old_full[16];
     uint32_t tmem_base;
     int abort;
     int epi_go[4];
@@ -83,14 +83,17 @@ struct K1Smem {                            // barriers and scalars, placed after
 
 __global__ void __launch_bounds__(K1_MAX_THREADS, 1)
 compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__ items, const __grid_constant__ SeedTable seeds,
-                   int seed_base, int r, float scale, float a, float b, int T, int stages, int S, int GW, int P, int late_wait)
+                   int seed_base, int r, float scale, float a, float b, int T, int gstages, int astages, int S, int GW, int P, int late_wait)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
     const int r_pad = (r + 15) & ~15;
     const uint32_t a_bytes = (uint32_t)r_pad * 128u;
-    const uint32_t stage_bytes = (uint32_t)T * G_TILE_BYTES + a_bytes;
-    K1Smem* ctl = reinterpret_cast<K1Smem*>(smem_raw + (smem_base - ptx::smem_addr(smem_raw)) + (size_t)stages * stage_bytes);
+    // two rings: G tiles (gstages x T tiles; the loads come from HBM and want many bytes in flight) and A tiles
+    // (astages x r_pad rows; produced on chip).  Each has its own full / empty barriers.
+    const uint32_t g_bytes = (uint32_t)T * G_TILE_BYTES;
+    const uint32_t a_ring = smem_base + (uint32_t)gstages * g_bytes;
+    K1Smem* ctl = reinterpret_cast<K1Smem*>(smem_raw + (a_ring - ptx::smem_addr(smem_raw)) + (size_t)astages * a_bytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     ptx::grid_launch_dependents();
@@ -100,11 +103,14 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
     while ((int)tmem_cols < T * r_pad) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < stages; ++s) {
+        for (int s = 0; s < gstages; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->full_g[s]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctl->empty_g[s]), 1);                   // this CTA's MMAs have consumed the G tiles
+        }
+        for (int s = 0; s < astages; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->full_a[s]), S > 1 ? 1 : GW / P);   // cluster: one arrival + the peers' bytes
             ptx::mbar_init(ptx::smem_addr(&ctl->slice_ready[s]), GW / P);
-            ptx::mbar_init(ptx::smem_addr(&ctl->empty[s]), S);                   // every CTA of the cluster has consumed the stage
+            ptx::mbar_init(ptx::smem_addr(&ctl->empty_a[s]), S);                   // every CTA of the cluster has consumed the A tile
         }
         ptx::mbar_init(ptx::smem_addr(&ctl->acc_full), 1);
         for (int k = 0; k < 16; ++k) ptx::mbar_init(ptx::smem_addr(&ctl->old_full[k]), 1);
@@ -120,9 +126,9 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
     // rows r .. r_pad of every A tile stay zero for the whole kernel
     if (r_pad > r) {
         const int pad_chunks = (r_pad - r) * 8;
-        for (int s = 0; s < stages; ++s)
+        for (int s = 0; s < astages; ++s)
             for (int t = threadIdx.x; t < pad_chunks; t += (int)blockDim.x)
-                ptx::st_shared_v4(smem_base + s * stage_bytes + T * G_TILE_BYTES + (uint32_t)r * 128u + t * 16u, 0, 0, 0, 0);
+                ptx::st_shared_v4(a_ring + s * a_bytes + (uint32_t)r * 128u + t * 16u, 0, 0, 0, 0);
         ptx::fence_proxy_async_smem();
     }
     ptx::tc_fence_before_sync();
@@ -143,21 +149,18 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
             ptx::prefetch_tensormap(&mat->map_g);
             int issued = 0;
             for (int ks = 0; ks < item.ksteps; ++ks) {
-                const int s = ks % stages, it = ks / stages;
-                if (!(S > 1 ? ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort)
-                            : ptx::mbar_wait(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort)))
-                    break;
+                const int s = ks % gstages, it = ks / gstages;
+                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->empty_g[s]), (it & 1) ^ 1, abort)) break;
                 const uint32_t bar = ptx::smem_addr(&ctl->full_g[s]);
                 ptx::mbar_arrive_expect_tx(bar, (uint32_t)item.tiles * G_TILE_BYTES);
                 for (int t = 0; t < item.tiles; ++t)
-                    ptx::tma_load_2d(smem_base + s * stage_bytes + t * G_TILE_BYTES, &mat->map_g, (item.kstep0 + ks) * 64,
-                                     item.row0 + t * 128, bar);
+                    ptx::tma_load_2d(smem_base + s * g_bytes + t * G_TILE_BYTES, &mat->map_g, (item.kstep0 + ks) * 64, item.row0 + t * 128, bar);
                 issued = ks + 1;
             }
             if (*abort) {
                 // nobody consumes any more: wait (bounded) until the copies still in flight have landed
-                for (int ks = max(0, issued - stages); ks < issued; ++ks)
-                    ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[ks % stages]), (ks / stages) & 1, abort);
+                for (int ks = max(0, issued - gstages); ks < issued; ++ks)
+                    ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[ks % gstages]), (ks / gstages) & 1, abort);
             }
         }
     } else if (warp == 1) {
@@ -167,23 +170,25 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
             const uint64_t desc_base = ptx::umma_desc_k_sw128(smem_base);
             bool ok = true;
             for (int ks = 0; ks < item.ksteps && ok; ++ks) {
-                const int s = ks % stages, it = ks / stages;
-                ok = (item.tiles == 0 || ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[s]), it & 1, abort)) &&
-                     (S > 1 ? ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->full_a[s]), it & 1, abort)
-                            : ptx::mbar_wait(ptx::smem_addr(&ctl->full_a[s]), it & 1, abort));
+                const int sg = ks % gstages, sa = ks % astages;
+                const uint32_t pa = (uint32_t)(ks / astages) & 1u;
+                ok = (item.tiles == 0 || ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[sg]), (uint32_t)(ks / gstages) & 1u, abort)) &&
+                     (S > 1 ? ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->full_a[sa]), pa, abort)
+                            : ptx::mbar_wait(ptx::smem_addr(&ctl->full_a[sa]), pa, abort));
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 // descriptors differ from the ring base only in the start-address field (16-byte units)
-                const uint64_t dstage = desc_base + (uint64_t)((s * stage_bytes) >> 4);
-                const uint64_t da_tile = dstage + (uint64_t)((T * G_TILE_BYTES) >> 4);
+                const uint64_t dstage = desc_base + (uint64_t)((sg * g_bytes) >> 4);
+                const uint64_t da_tile = desc_base + (uint64_t)((a_ring - smem_base + sa * a_bytes) >> 4);
                 for (int t = 0; t < item.tiles; ++t) {
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
                         ptx::umma_bf16(tmem + t * r_pad, dstage + (uint64_t)((t * G_TILE_BYTES + kk * 32) >> 4), da_tile + (uint64_t)(kk * 2), idesc,
                                        (ks | kk) != 0);
                 }
-                // the stage is free once every CTA of the cluster has consumed its copy of the A tile
-                const uint32_t ebar = ptx::smem_addr(&ctl->empty[s]);
+                if (item.tiles > 0) ptx::umma_commit(ptx::smem_addr(&ctl->empty_g[sg]));
+                // the A stage is free once every CTA of the cluster has consumed its copy of the tile
+                const uint32_t ebar = ptx::smem_addr(&ctl->empty_a[sa]);
                 if (S == 1) ptx::umma_commit(ebar);
                 else if (item.tiles > 0) ptx::umma_commit_cluster(ebar, (uint16_t)((1u << S) - 1u));
                 else
@@ -196,10 +201,10 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
         if (lane == 0 && S > 1) {
             const uint32_t slice_bytes = (uint32_t)(r_pad / S) * 128u;
             for (int ks = 0; ks < item.ksteps; ++ks) {
-                const int s = ks % stages, it = ks / stages;
+                const int s = ks % astages, it = ks / astages;
                 if (!ptx::mbar_wait(ptx::smem_addr(&ctl->slice_ready[s]), it & 1, abort)) break;
                 const uint32_t fbar = ptx::smem_addr(&ctl->full_a[s]);
-                const uint32_t src = smem_base + s * stage_bytes + T * G_TILE_BYTES + rank * slice_bytes;
+                const uint32_t src = a_ring + s * a_bytes + rank * slice_bytes;
                 ptx::mbar_arrive_expect_tx(fbar, (uint32_t)(S - 1) * slice_bytes);   // own slice is in place; peers' bytes to come
                 for (int d = 0; d < S; ++d)
                     if (d != (int)rank) ptx::bulk_copy_to_peer(ptx::map_to_cta(src, d), src, slice_bytes, ptx::map_to_cta(fbar, d));
@@ -217,11 +222,11 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
         const int tasks = r * 8;                              // (row j, 16-byte chunk c) pairs of one A tile
         bool ok = true;
         for (int ks = team; ks < item.ksteps && ok; ks += P) {
-            const int s = ks % stages, it = ks / stages;
-            ok = S > 1 ? ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort)
-                       : ptx::mbar_wait(ptx::smem_addr(&ctl->empty[s]), (it & 1) ^ 1, abort);
+            const int s = ks % astages, it = ks / astages;
+            ok = S > 1 ? ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->empty_a[s]), (it & 1) ^ 1, abort)
+                       : ptx::mbar_wait(ptx::smem_addr(&ctl->empty_a[s]), (it & 1) ^ 1, abort);
             if (!ok) break;
-            const uint32_t a_tile = smem_base + s * stage_bytes + T * G_TILE_BYTES;
+            const uint32_t a_tile = a_ring + s * a_bytes;
             const uint32_t q0 = (uint32_t)(item.kstep0 + ks) * 16u;
             if (S == 1) {
                 for (int t = g; t < tasks; t += team_threads) {
@@ -260,10 +265,10 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
         //         a bulk reduction, nothing is read back;
         //   store S <- a*acc       (b == 0 and the item owns its rows);
         //   rmw   S <- b*S + a*acc (the item owns its rows): the old chunk comes in by a bulk load, one chunk ahead.
-        // The chunk buffers are the tiles of the ring, which nothing uses once the last MMA has completed.
+        // The chunk buffers are the tiles of the G ring, which nothing uses once the last MMA has completed (the A ring is
+        // left alone: this CTA's last slices may still be on their way to the peers).
         const int gw = warp - 2;
-        const int slots_per_stage = T + (int)(a_bytes / (uint32_t)G_TILE_BYTES);   // 16 KB areas of one stage
-        const int areas = stages * slots_per_stage;
+        const int areas = gstages * T;                            // 16 KB areas: the tiles of the G ring
         const int EG = min(min(GW >> 2, 4), areas);               // groups at work
         if (gw < 4 * EG && item.tiles > 0) {
             const int grp = gw >> 2;
@@ -280,8 +285,7 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
             const int total = item.tiles * nchunks;               // chunks of this CTA; the group takes grp, grp + EG, ...
             const int NB = min(areas / EG, 4);                    // buffers of this group
             auto buffer = [&](int u) {                            // u: running index of the group's chunks
-                const int k = grp * NB + u % NB;
-                return smem_base + (uint32_t)(k / slots_per_stage) * stage_bytes + (uint32_t)(k % slots_per_stage) * G_TILE_BYTES;
+                return smem_base + (uint32_t)(grp * NB + u % NB) * G_TILE_BYTES;
             };
             auto wait_reads = [&]() {                             // all but the newest NB-2 stores have been read out of shared memory
                 if (NB >= 4) ptx::tma_store_wait_read<2>();

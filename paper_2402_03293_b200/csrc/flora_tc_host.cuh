@@ -23,7 +23,7 @@ struct TcSet {
     bool decompress_ready = false;
     bool transient = false;             // device buffers come from the stream-ordered allocator
     int count = 0, r = 0;
-    int T = 1, stages = 2, S = 1, GW = 8, P = 1;
+    int T = 1, gstages = 2, astages = 2, S = 1, GW = 8, P = 1;
     std::vector<int> k1_launch_first_mat;
     size_t k1_smem = 0;
     TcMatrix* d_mats = nullptr;
@@ -173,8 +173,17 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
     // overlaps the loads of the other (single-CTA clusters only)
     int per_sm = (S == 1 && cols <= 256 && 2 * stage <= SMEM_BUDGET / 2) ? 2 : 1;
     per_sm = tune_knob("FLORA_K1_PER_SM", per_sm, 1, (S == 1 && cols <= 256) ? 2 : 1);
-    int stages = (int)std::min<size_t>(8, SMEM_BUDGET / per_sm / stage);
-    stages = tune_knob("FLORA_K1_STAGES", stages, 1, std::max(1, stages));
+    // Two rings.  The G tiles come from HBM: with a latency near 2 us under load, the bytes in flight per SM, not the
+    // link, bound the intake, so the G ring gets all the shared memory the A ring does not need.  A tiles are made on
+    // chip: two stages; three (four for the large tiles of ranks above 128) where slices travel between the CTAs of a
+    // cluster and the slowest CTA paces all of them.
+    const size_t g_stage = (size_t)T * G_TILE_BYTES, a_stage = (size_t)r_pad * 128;
+    const size_t ring_budget = SMEM_BUDGET / per_sm - sizeof(K1Smem) - 1024;
+    int astages = S > 1 ? (r_pad > 128 ? 4 : 3) : 2;
+    if ((ring_budget - astages * a_stage) / g_stage < 2) astages = 2;
+    astages = tune_knob("FLORA_K1_ASTAGES", astages, 1, 8);
+    int gstages = (int)std::min<size_t>(8, (ring_budget - std::min(ring_budget, astages * a_stage)) / g_stage);
+    gstages = tune_knob("FLORA_K1_GSTAGES", std::max(1, gstages), 1, std::max(1, gstages));
     // generator warps: 16 where one CTA owns the SM and generation is a sizeable share of the work
     int GW = (per_sm == 1 && ratio / S > 0.15) ? 16 : 8;
     GW = tune_knob("FLORA_K1_GEN_WARPS", GW, 4, per_sm == 1 ? K1_MAX_GEN_WARPS : 8);
@@ -183,15 +192,16 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
     {
         const int tile_tasks = (S > 1 ? r_pad / S : r) * 8;
         int P = 1;
-        while (2 * P <= stages && GW % (2 * P) == 0 && 32 * GW / (2 * P) >= tile_tasks) P *= 2;
+        while (2 * P <= astages && GW % (2 * P) == 0 && 32 * GW / (2 * P) >= tile_tasks) P *= 2;
         P = tune_knob("FLORA_K1_TEAMS", P, 1, 8);
-        while (P > 1 && (GW % P || P > stages || (P & (P - 1)))) --P;
+        while (P > 1 && (GW % P || P > astages || (P & (P - 1)))) --P;
         set.P = P;
     }
     set.T = T;
     set.S = S;
-    set.stages = stages;
-    set.k1_smem = (size_t)stages * stage + sizeof(K1Smem) + 1024;
+    set.gstages = gstages;
+    set.astages = astages;
+    set.k1_smem = (size_t)gstages * g_stage + (size_t)astages * a_stage + sizeof(K1Smem) + 1024;
     // column chunks: aim at about `waves` items per slot (a slot is a CTA, or a cluster), at least 8 steps each
     int64_t slots = std::max<int64_t>(1, (int64_t)sm_count() * per_sm / S);
     if (cudaFuncSetAttribute(compress_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)set.k1_smem) != cudaSuccess) cudaGetLastError();
@@ -624,7 +634,7 @@ inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, 
         cfg.numAttrs = set.S > 1 ? 2 : 1;
         const TcMatrix* mats = set.d_mats;
         const K1Item* items = set.d_k1 + begin;
-        if (cudaLaunchKernelEx(&cfg, compress_tc_kernel, mats, items, table, seed_base, r, scale, a, b, set.T, set.stages, set.S, set.GW, set.P, l == 0 ? late_wait : 0) !=
+        if (cudaLaunchKernelEx(&cfg, compress_tc_kernel, mats, items, table, seed_base, r, scale, a, b, set.T, set.gstages, set.astages, set.S, set.GW, set.P, l == 0 ? late_wait : 0) !=
             cudaSuccess)
             return FLORA_ERR_CUDA;
         launches.fetch_add(1, std::memory_order_relaxed);
