@@ -91,14 +91,14 @@ flora_status flora_momentum_step(const flora_mat* G, flora_mat* M, float beta, u
 /* Algorithm 2, resampling branch:  M <- M A(seed_old) A(seed_new)^T, evaluated as M (A_old A_new^T).
  * M: n x r f32, in place.  `m` is the column count of the weight matrix (A is r x m) and
  * `operand` the dtype of the gradients that were compressed into M (it fixes the precision of A).
- * Uses r*r floats of scratch taken from the stream-ordered allocator (cudaMallocAsync) and
- * returned to it before the call returns; FLORA_ERR_ALLOC if that fails. */
+ * Uses r*r floats of scratch taken from a stream-ordered memory pool that the library owns (one per device,
+ * created at the first such call) and returned to it before the call returns; FLORA_ERR_ALLOC if that fails. */
 flora_status flora_resample_transfer(flora_mat* M, int64_t m, int32_t operand, uint64_t seed_old, uint64_t seed_new, void* stream);
 
 /* The same operation as flora_resample_transfer for callers that must not allocate.  (The paper has no
  * counterpart to this call: it is a packaging of Algorithm 2's transfer for a constrained caller.)
  *
- * flora_resample_transfer borrows its r x r scratch from cudaMallocAsync.  That is unusable for code that
+ * flora_resample_transfer borrows its r x r scratch from a stream-ordered allocation.  That is unusable for code that
  * runs after all device memory has been handed out (an inference or training process whose memory plan is
  * fixed up front and which treats any later allocation as a failure), for code that may not touch the
  * allocator at all at this point (a latency-critical loop, a thread that does not own the memory pool), and

@@ -16,6 +16,7 @@
 #include "../../include/flora.h"
 #include "flora_rng.cuh"
 #include "flora_simt.cuh"
+#include "flora_pool.cuh"
 #include "flora_tc_host.cuh"
 #include "flora_gram.cuh"
 
@@ -236,7 +237,7 @@ flora_status flora_transfer_axpby(flora_mat* dst, const flora_mat* src, int64_t 
         if (dst->rows <= 0x7FFFFFFF && m <= 0x7FFFFFFF) return transfer_tc(jobs, r, a, b, as_stream(stream), g_launches);
     }
     float* T = nullptr;
-    if (cudaMallocAsync((void**)&T, sizeof(float) * r * r, as_stream(stream)) != cudaSuccess) {
+    if (scratch_alloc((void**)&T, sizeof(float) * r * r, as_stream(stream)) != cudaSuccess) {
         cudaGetLastError();
         return FLORA_ERR_ALLOC;
     }
@@ -404,7 +405,7 @@ flora_status flora_set_resample_transfer(flora_set* set, const uint64_t* seeds_o
         }
         return transfer_tc(jobs, r, 1.0f, 0.0f, as_stream(stream), g_launches);
     }
-    if (cudaMallocAsync((void**)&T, sizeof(float) * r * r, as_stream(stream)) != cudaSuccess) {
+    if (scratch_alloc((void**)&T, sizeof(float) * r * r, as_stream(stream)) != cudaSuccess) {
         cudaGetLastError();
         return FLORA_ERR_ALLOC;
     }
@@ -492,7 +493,7 @@ flora_status flora_device_status(void)
 flora_status flora_debug_wait_timeout_selftest(void* stream)
 {
     int* flag = nullptr;
-    if (cudaMallocAsync((void**)&flag, sizeof(int), as_stream(stream)) != cudaSuccess) {
+    if (scratch_alloc((void**)&flag, sizeof(int), as_stream(stream)) != cudaSuccess) {
         cudaGetLastError();
         return FLORA_ERR_ALLOC;
     }

@@ -17,6 +17,7 @@
 #include <vector>
 
 #include "../../include/flora.h"
+#include "flora_pool.cuh"
 #include "flora_ptx.cuh"
 #include "flora_rng.cuh"
 
@@ -385,7 +386,7 @@ inline flora_status transfer_tc(std::vector<GramJob>& jobs, int r, float a, floa
     }
     const size_t tables_off = t_bytes * jobs.size();
     uint8_t* buf = nullptr;
-    if (cudaMallocAsync((void**)&buf, tables_off + tables.size(), st) != cudaSuccess) {
+    if (scratch_alloc((void**)&buf, tables_off + tables.size(), st) != cudaSuccess) {
         cudaGetLastError();
         return FLORA_ERR_ALLOC;
     }

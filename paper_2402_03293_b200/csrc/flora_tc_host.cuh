@@ -11,6 +11,7 @@
 #include <atomic>
 #include <vector>
 
+#include "flora_pool.cuh"
 #include "flora_tc.cuh"
 
 namespace flora {
@@ -467,7 +468,7 @@ inline flora_status upload(T** dst, const std::vector<T>& src, bool transient, c
     if (src.empty()) return FLORA_OK;
     const size_t bytes = src.size() * sizeof(T);
     if (!*dst) {
-        cudaError_t e = transient ? cudaMallocAsync((void**)dst, bytes, st) : cudaMalloc((void**)dst, bytes);
+        cudaError_t e = transient ? scratch_alloc((void**)dst, bytes, st) : cudaMalloc((void**)dst, bytes);
         if (e != cudaSuccess) {
             cudaGetLastError();
             return FLORA_ERR_ALLOC;
@@ -526,7 +527,7 @@ inline flora_status tc_set_build_on(TcSet& set, const std::vector<flora_mat>& G,
                 total += (((size_t)S[i].rows * k_pad * 2) + 1023) & ~(size_t)1023;
             }
             if (total) {
-                cudaError_t e = transient ? cudaMallocAsync((void**)&set.d_sb, total, st) : cudaMalloc((void**)&set.d_sb, total);
+                cudaError_t e = transient ? scratch_alloc((void**)&set.d_sb, total, st) : cudaMalloc((void**)&set.d_sb, total);
                 if (e != cudaSuccess) {
                     cudaGetLastError();
                     return FLORA_ERR_ALLOC;
