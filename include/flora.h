@@ -183,6 +183,17 @@ flora_status flora_set_read_weights_to_host(flora_set* set, void* const* host_W,
 /* Test hook: 0 = choose the kernel automatically (tensor-core kernels when dtype, alignment and
  * rank allow), 1 = always the plain fp32 SIMT kernels.  Process-wide. */
 void flora_debug_force_path(int path);
+
+/* Test hook for the host-side work decomposition of the tensor-core kernels (no kernel is launched; works without a
+ * GPU, in which case 148 SMs and an unconstrained cluster residency are assumed).  `rows`/`cols`: the shapes of
+ * `count` bf16 matrices; `r`: the rank.  which = 0: the compression kernel; items are 6 x int32 {matrix, first row,
+ * 128-row tiles, first 64-column step, steps, owns-its-rows flag}; params (8 x int32) = {tiles per CTA T, cluster
+ * size S, G stages, A stages, generator warps, teams, launches, shared memory bytes}.  which = 1: the decompression
+ * kernel; items are 4 x int32 {matrix, first column, first row, 128-row tiles}; params = {slab width bn, W slots,
+ * S chunk stages, slab buffers, generator warps, bf16-sketch flag, launches, shared memory bytes}.  At most
+ * `capacity` items are written (host memory, caller-owned); *n_items receives the full count. */
+flora_status flora_debug_plan(const int64_t* rows, const int64_t* cols, int64_t count, int32_t r, int32_t which, int32_t* items, int64_t capacity,
+                              int64_t* n_items, int32_t* params);
 /* Kernels launched by this library since load (your own count of launches). */
 uint64_t flora_launch_count(void);
 /* Reads (synchronously, with a device->host copy) and clears the device-side error word that

@@ -29,7 +29,7 @@ EXPORTS = [
     "flora_set_rebind_gradients", "flora_set_compress_accumulate", "flora_set_momentum_step",
     "flora_set_decompress_apply", "flora_set_resample_transfer", "flora_set_zero_state", "flora_derive_seed",
     "flora_resamples_at", "flora_set_compress_accumulate_from_host", "flora_set_read_weights_to_host",
-    "flora_debug_force_path", "flora_debug_wait_timeout_selftest", "flora_launch_count", "flora_device_status", "flora_status_string", "flora_version",
+    "flora_debug_force_path", "flora_debug_plan", "flora_debug_wait_timeout_selftest", "flora_launch_count", "flora_device_status", "flora_status_string", "flora_version",
 ]
 
 
@@ -77,6 +77,7 @@ def load() -> ctypes.CDLL:
             "flora_set_compress_accumulate_from_host": (I32, [P, ctypes.POINTER(P), ctypes.POINTER(U64), P]),
             "flora_set_read_weights_to_host": (I32, [P, ctypes.POINTER(P), P]),
             "flora_debug_force_path": (None, [ctypes.c_int]),
+            "flora_debug_plan": (I32, [P, P, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, P, ctypes.c_int64, P, P]),
             "flora_debug_wait_timeout_selftest": (I32, [P]),
             "flora_launch_count": (U64, []),
             "flora_device_status": (I32, []),
@@ -190,6 +191,25 @@ def flora_resamples_at(t: int, kappa: int) -> bool:
 
 def flora_debug_force_path(path: int) -> None:
     load().flora_debug_force_path(path)
+
+
+def flora_debug_plan(shapes, r: int, which: str):
+    """Work items and launch parameters the library would use for bf16 matrices of these (rows, cols) shapes.
+
+    which = "compress" or "decompress".  Returns (items, params): items as a list of tuples, params as a tuple of
+    eight ints (see include/flora.h).  No kernel runs; usable without a GPU."""
+    count = len(shapes)
+    rows = (ctypes.c_int64 * max(count, 1))(*[int(n) for n, _ in shapes])
+    cols = (ctypes.c_int64 * max(count, 1))(*[int(m) for _, m in shapes])
+    w = 0 if which == "compress" else 1
+    width = 6 if w == 0 else 4
+    n = ctypes.c_int64(0)
+    params = (ctypes.c_int32 * 8)()
+    _check(load().flora_debug_plan(rows, cols, count, r, w, None, 0, ctypes.byref(n), params), "flora_debug_plan")
+    buf = (ctypes.c_int32 * max(1, n.value * width))()
+    _check(load().flora_debug_plan(rows, cols, count, r, w, buf, n.value, ctypes.byref(n), params), "flora_debug_plan")
+    items = [tuple(buf[i * width + j] for j in range(width)) for i in range(n.value)]
+    return items, tuple(params)
 
 
 def flora_debug_wait_timeout_selftest(stream=None) -> int:

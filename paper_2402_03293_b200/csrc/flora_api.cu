@@ -481,6 +481,47 @@ int flora_resamples_at(int64_t t, int64_t kappa) { return (kappa > 0 && t >= 0 &
 // diagnostics
 // ------------------------------------------------------------------------------------------------
 void flora_debug_force_path(int path) { g_force_path.store(path == 1 ? 1 : 0); }
+
+flora_status flora_debug_plan(const int64_t* rows, const int64_t* cols, int64_t count, int32_t r, int32_t which, int32_t* items, int64_t capacity,
+                              int64_t* n_items, int32_t* params)
+{
+    if (!rows || !cols || !n_items || !params || (capacity > 0 && !items)) return FLORA_ERR_NULL;
+    if (count < 0 || capacity < 0) return FLORA_ERR_SHAPE;
+    if (r < 1 || r > 256) return FLORA_ERR_RANK;
+    std::vector<flora_mat> mats((size_t)count);
+    for (int64_t i = 0; i < count; ++i) {
+        if (rows[i] < 0 || cols[i] < 0 || rows[i] > 0x7FFFFF00ll || cols[i] > 0x7FFFFF00ll) return FLORA_ERR_SHAPE;
+        mats[(size_t)i] = flora_mat{nullptr, rows[i], cols[i], cols[i], FLORA_BF16};
+    }
+    TcSet set;
+    set.count = (int)count;
+    set.r = r;
+    const int width = which == 0 ? 6 : 4;
+    if (which == 0) {
+        plan_compress(set, mats, r);
+        *n_items = (int64_t)set.h_k1.size();
+        const int32_t p[8] = {set.T, set.S, set.gstages, set.astages, set.GW, set.P, (int32_t)(set.k1_launch_begin.size() - 1), (int32_t)set.k1_smem};
+        memcpy(params, p, sizeof(p));
+        for (int64_t i = 0; i < std::min<int64_t>(*n_items, capacity); ++i) {
+            const K1Item& it = set.h_k1[(size_t)i];
+            const int32_t v[6] = {it.mat, it.row0, it.tiles, it.kstep0, it.ksteps, it.direct};
+            memcpy(items + i * width, v, sizeof(v));
+        }
+    } else {
+        plan_decompress(set, mats, r);
+        *n_items = (int64_t)set.h_k2.size();
+        const int32_t p[8] = {set.bn, set.slots, set.cstages, set.k2_nslabs, set.k2_gw, set.k2_bf16 ? 1 : 0, (int32_t)(set.k2_launch_begin.size() - 1),
+                              (int32_t)set.k2_smem};
+        memcpy(params, p, sizeof(p));
+        for (int64_t i = 0; i < std::min<int64_t>(*n_items, capacity); ++i) {
+            const K2Item& it = set.h_k2[(size_t)i];
+            const int32_t v[4] = {it.mat, it.col0, it.row0, it.tiles};
+            memcpy(items + i * width, v, sizeof(v));
+        }
+    }
+    cudaGetLastError();        // without a device the occupancy queries inside the planners fail and fall back; leave no sticky error
+    return FLORA_OK;
+}
 uint64_t flora_launch_count(void) { return g_launches.load(); }
 
 flora_status flora_device_status(void)
