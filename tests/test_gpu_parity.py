@@ -309,3 +309,31 @@ def test_bounded_wait_gives_up_and_reports_a_timeout():
     G = _g(256, 512, "bf16", 3)
     fb.flora_compress_accumulate(G, C, 5, 8)
     assert rel_err(C.cpu().numpy(), oracle_compress(G, torch.zeros(256, 8), 5)) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("n,m,r", [(2048, 2304, 32), (4096, 1024, 128), (1600, 1600, 256), (768, 3072, 64)])
+def test_repeated_launches_are_bit_identical(n, m, r):
+    """Race detector: the same call, repeated, must give the same bits wherever the arithmetic fixes the order of
+    the additions (decompression always; compression when every row of the sketch has a single owner)."""
+    G = _g(n, m, "bf16", 11)
+    items, _ = fb.flora_debug_plan([(n, m)], r, "compress")
+    owned = all(it[5] == 1 for it in items)
+    first_c = first_m = first_w = None
+    W0 = (torch.randn(n, m, device=DEV) * 0.02).to(torch.bfloat16)
+    S = torch.randn(n, r, device=DEV)
+    for it in range(25):
+        C = torch.zeros(n, r, device=DEV)
+        fb.flora_compress_accumulate(G, C, 9, r)
+        M = torch.ones(n, r, device=DEV)
+        fb.flora_momentum_step(G, M, 0.75, 9)
+        W = W0.clone()
+        fb.flora_decompress_apply(W, S, 9, 0.5, 1.0)
+        if it == 0:
+            first_c, first_m, first_w = C, M, W
+        else:
+            assert torch.equal(W, first_w)
+            if owned:
+                assert torch.equal(C, first_c) and torch.equal(M, first_m)
+            else:
+                assert rel_err(C.cpu().numpy(), first_c.cpu().numpy()) <= 1e-5
+    assert fb.flora_device_status() == 0
