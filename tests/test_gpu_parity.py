@@ -250,29 +250,37 @@ def test_host_to_device_entry_points():
 # --------------------------------------------------------------------------------------- full-size configs, sampled rows
 @pytest.mark.parametrize("name", ["gpt2_small_set"])
 def test_full_size_set_sampled_rows(name):
+    """The benchmark's step at full size and in its launch configuration: tau gradient sets bound to one set of weights
+    and sketches, tau compressions, one decompress-apply with scale 1/tau, the reset of C; sampled rows replayed on the oracle."""
     w = wl.WORKLOADS[name]
     count = len(w.shapes)
-    G = [wl.gradient(w, i, 0, device=DEV) for i in range(count)]
+    G = [[wl.gradient(w, i, k, device=DEV) for i in range(count)] for k in range(w.tau)]
     W = [wl.weight(w, i, device=DEV, std=0.02) for i in range(count)]
     W0 = [x.clone() for x in W]
     S = [torch.zeros(n, w.r, device=DEV) for n, _ in w.shapes]
-    fset = fb.FloraSet(G, W, S)
+    sets = [fb.FloraSet(G[k], W, S) for k in range(w.tau)]
     seeds = [fb.flora_derive_seed(3, i, 0) for i in range(count)]
-    fset.compress_accumulate(seeds)
-    fset.compress_accumulate(seeds)
-    fset.decompress_apply(seeds, 4.0, 0.5)
+    for k in range(w.tau):
+        sets[k].compress_accumulate(seeds)
+    Sacc = [x.clone() for x in S]
+    sets[0].decompress_apply(seeds, 4.0, 1.0 / w.tau)
+    sets[0].zero_state()
     torch.cuda.synchronize()
+    assert fb.flora_device_status() == 0
     for i in range(0, count, 5):
         n, m = w.shapes[i]
         rows = sample_rows(n, 24, i)
-        Gr = G[i][torch.from_numpy(rows).to(DEV)].cpu()
-        c1 = oracle_compress(Gr, torch.zeros(len(rows), w.r), seeds[i])
-        c2 = oracle_compress(Gr, torch.from_numpy(c1), seeds[i])
-        got = S[i].cpu().numpy()[rows]
-        assert rel_err(got, c2) <= TOL["bf16"], i
-        ref = oracle_decompress(W0[i][torch.from_numpy(rows).to(DEV)].cpu(), torch.from_numpy(got), seeds[i], 4.0, 0.5)
+        idx = torch.from_numpy(rows).to(DEV)
+        c = np.zeros((len(rows), w.r), dtype=np.float32)
+        for k in range(w.tau):
+            c = oracle_compress(G[k][i][idx].cpu(), torch.from_numpy(c), seeds[i])
+        got = Sacc[i].cpu().numpy()[rows]
+        assert rel_err(got, c) <= TOL["bf16"], i
+        ref = oracle_decompress(W0[i][idx].cpu(), torch.from_numpy(got), seeds[i], 4.0, 1.0 / w.tau)
         assert rel_err(values(wl.as_numpy(W[i])[rows]), values(ref)) <= TOL["bf16"], i
-    fset.close()
+        assert not S[i].any()                                                      # C is zero again for the next cycle
+    for s_ in sets:
+        s_.close()
 
 
 # --------------------------------------------------------------------------------------- robustness
