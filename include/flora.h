@@ -95,6 +95,13 @@ flora_status flora_momentum_step(const flora_mat* G, flora_mat* M, float beta, u
  * created at the first such call) and returned to it before the call returns; FLORA_ERR_ALLOC if that fails. */
 flora_status flora_resample_transfer(flora_mat* M, int64_t m, int32_t operand, uint64_t seed_old, uint64_t seed_new, void* stream);
 
+/* Algorithm 2 at a step where the projection is resampled, as one call:
+ *      M <- beta * (M A(seed_old) A(seed_new)^T) + (1 - beta) * G A(seed_new)^T.
+ * Equal (up to rounding order) to flora_resample_transfer followed by flora_momentum_step with seed_new, but the
+ * factor beta rides on the transfer's last pass over M and the compression then only adds: M is read and written
+ * once less.  G: n x m (f32 or bf16), M: n x r f32, in place.  Scratch and errors as for flora_resample_transfer. */
+flora_status flora_momentum_step_resampled(const flora_mat* G, flora_mat* M, float beta, uint64_t seed_old, uint64_t seed_new, void* stream);
+
 /* The same operation as flora_resample_transfer for callers that must not allocate.  (The paper has no
  * counterpart to this call: it is a packaging of Algorithm 2's transfer for a constrained caller.)
  *
@@ -153,6 +160,8 @@ flora_status flora_set_compress_accumulate(flora_set* set, const uint64_t* seeds
 flora_status flora_set_momentum_step(flora_set* set, float beta, const uint64_t* seeds, void* stream);
 flora_status flora_set_decompress_apply(flora_set* set, const uint64_t* seeds, float lr, float scale, void* stream);
 flora_status flora_set_resample_transfer(flora_set* set, const uint64_t* seeds_old, const uint64_t* seeds_new, void* stream);
+/* flora_momentum_step_resampled for every matrix of the set (created with gradients). */
+flora_status flora_set_momentum_step_resampled(flora_set* set, float beta, const uint64_t* seeds_old, const uint64_t* seeds_new, void* stream);
 /* Sets every sketch of the set to zero (start of an accumulation cycle, Algorithm 1). */
 flora_status flora_set_zero_state(flora_set* set, void* stream);
 

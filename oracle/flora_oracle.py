@@ -174,6 +174,13 @@ def resample_transfer(M: np.ndarray, A_old: np.ndarray, A_new: np.ndarray) -> No
         raise MemoryError("oracle transfer")
 
 
+def momentum_step_resampled(G: np.ndarray, A_old: np.ndarray, A_new: np.ndarray, beta: float, M: np.ndarray) -> None:
+    """Algorithm 2 at a resampling step, in the paper's order: first M <- (M A_old) A_new^T, then
+    M <- beta M + (1 - beta) G A_new^T (in place on M)."""
+    resample_transfer(M, A_old, A_new)
+    momentum_step(G, A_new, beta, M)
+
+
 def transfer_axpby(dst: np.ndarray, src: np.ndarray, A_old: np.ndarray, A_new: np.ndarray,
                    a: float, b: float) -> None:
     """dst <- b dst + a (src A_old) A_new^T: Algorithm 1's output fed to Algorithm 2's update."""

@@ -24,10 +24,10 @@ FLORA_F32, FLORA_BF16 = 0, 1
 
 # every symbol include/flora.h declares
 EXPORTS = [
-    "flora_compress_accumulate", "flora_decompress_apply", "flora_momentum_step", "flora_resample_transfer",
+    "flora_compress_accumulate", "flora_decompress_apply", "flora_momentum_step", "flora_momentum_step_resampled", "flora_resample_transfer",
     "flora_resample_transfer_static", "flora_transfer_axpby", "flora_materialize_A", "flora_set_create", "flora_set_destroy",
     "flora_set_rebind_gradients", "flora_set_compress_accumulate", "flora_set_momentum_step",
-    "flora_set_decompress_apply", "flora_set_resample_transfer", "flora_set_zero_state", "flora_derive_seed",
+    "flora_set_decompress_apply", "flora_set_resample_transfer", "flora_set_momentum_step_resampled", "flora_set_zero_state", "flora_derive_seed",
     "flora_resamples_at", "flora_set_compress_accumulate_from_host", "flora_set_read_weights_to_host",
     "flora_debug_force_path", "flora_debug_plan", "flora_debug_wait_timeout_selftest", "flora_launch_count", "flora_device_status", "flora_status_string", "flora_version",
 ]
@@ -61,6 +61,7 @@ def load() -> ctypes.CDLL:
             "flora_decompress_apply": (I32, [MP, MP, U64, F, F, P]),
             "flora_momentum_step": (I32, [MP, MP, F, U64, P]),
             "flora_resample_transfer": (I32, [MP, I64, I32, U64, U64, P]),
+            "flora_momentum_step_resampled": (I32, [MP, MP, F, U64, U64, P]),
             "flora_resample_transfer_static": (I32, [MP, I64, I32, U64, U64, P]),
             "flora_transfer_axpby": (I32, [MP, MP, I64, I32, U64, U64, F, F, P]),
             "flora_materialize_A": (I32, [MP, U64, P]),
@@ -71,6 +72,7 @@ def load() -> ctypes.CDLL:
             "flora_set_momentum_step": (I32, [P, F, ctypes.POINTER(U64), P]),
             "flora_set_decompress_apply": (I32, [P, ctypes.POINTER(U64), F, F, P]),
             "flora_set_resample_transfer": (I32, [P, ctypes.POINTER(U64), ctypes.POINTER(U64), P]),
+            "flora_set_momentum_step_resampled": (I32, [P, F, ctypes.POINTER(U64), ctypes.POINTER(U64), P]),
             "flora_set_zero_state": (I32, [P, P]),
             "flora_derive_seed": (U64, [U64, U64, U64]),
             "flora_resamples_at": (ctypes.c_int, [I64, I64]),
@@ -152,6 +154,12 @@ def flora_momentum_step(G: torch.Tensor, M: torch.Tensor, beta: float, seed: int
     g, m_ = mat(G), mat(M)
     _check(load().flora_momentum_step(ctypes.byref(g), ctypes.byref(m_), beta, seed, _stream(stream)),
            "flora_momentum_step")
+
+
+def flora_momentum_step_resampled(G: torch.Tensor, M: torch.Tensor, beta: float, seed_old: int, seed_new: int, stream=None) -> None:
+    g, m_ = mat(G), mat(M)
+    _check(load().flora_momentum_step_resampled(ctypes.byref(g), ctypes.byref(m_), beta, seed_old, seed_new, _stream(stream)),
+           "flora_momentum_step_resampled")
 
 
 def flora_resample_transfer(M: torch.Tensor, m: int, operand, seed_old: int, seed_new: int, stream=None) -> None:
@@ -294,6 +302,10 @@ class FloraSet:
     def resample_transfer(self, seeds_old: Sequence[int], seeds_new: Sequence[int], stream=None) -> None:
         _check(load().flora_set_resample_transfer(self._h, _u64_array(seeds_old), _u64_array(seeds_new),
                                                   _stream(stream)), "flora_set_resample_transfer")
+
+    def momentum_step_resampled(self, beta: float, seeds_old: Sequence[int], seeds_new: Sequence[int], stream=None) -> None:
+        _check(load().flora_set_momentum_step_resampled(self._h, beta, _u64_array(seeds_old), _u64_array(seeds_new),
+                                                        _stream(stream)), "flora_set_momentum_step_resampled")
 
     def zero_state(self, stream=None) -> None:
         _check(load().flora_set_zero_state(self._h, _stream(stream)), "flora_set_zero_state")

@@ -215,6 +215,18 @@ flora_status flora_momentum_step(const flora_mat* G, flora_mat* M, float beta, u
     return simt_compress(G, M, seed, 1.0f - beta, beta, as_stream(stream));
 }
 
+flora_status flora_momentum_step_resampled(const flora_mat* G, flora_mat* M, float beta, uint64_t seed_old, uint64_t seed_new, void* stream)
+{
+    flora_status st = check_pair(G, M);
+    if (st) return st;
+    if (G->rows == 0) return FLORA_OK;
+    // M <- beta (M A_old A_new^T): the transfer's own scaling; then M <- M + (1 - beta) G A_new^T, a pure accumulation
+    st = flora_transfer_axpby(M, M, G->cols, G->dtype, seed_old, seed_new, beta, 0.0f, stream);
+    if (st) return st;
+    if (G->cols > 0 && use_tc_compress(G, M)) return tc_compress_single(G, M, seed_new, 1.0f - beta, 1.0f, as_stream(stream), g_launches);
+    return simt_compress(G, M, seed_new, 1.0f - beta, 1.0f, as_stream(stream));
+}
+
 flora_status flora_decompress_apply(flora_mat* W, const flora_mat* C, uint64_t seed, float lr, float scale, void* stream)
 {
     flora_status st = check_pair(W, C);
@@ -386,7 +398,7 @@ flora_status flora_set_decompress_apply(flora_set* set, const uint64_t* seeds, f
     return FLORA_OK;
 }
 
-flora_status flora_set_resample_transfer(flora_set* set, const uint64_t* seeds_old, const uint64_t* seeds_new, void* stream)
+static flora_status set_transfer(flora_set* set, const uint64_t* seeds_old, const uint64_t* seeds_new, float a, void* stream)
 {
     if (!set || !seeds_old || !seeds_new) return FLORA_ERR_NULL;
     const std::vector<flora_mat>& big = set->has_G ? set->G : set->W;
@@ -403,7 +415,7 @@ flora_status flora_set_resample_transfer(flora_set* set, const uint64_t* seeds_o
             jobs.push_back(GramJob{nullptr, (float*)set->S[i].data, (const float*)set->S[i].data, set->S[i].ld, set->S[i].ld,
                                    (int32_t)set->S[i].rows, (int32_t)big[i].cols, seeds_old[i], seeds_new[i]});
         }
-        return transfer_tc(jobs, r, 1.0f, 0.0f, as_stream(stream), g_launches);
+        return transfer_tc(jobs, r, a, 0.0f, as_stream(stream), g_launches);
     }
     if (scratch_alloc((void**)&T, sizeof(float) * r * r, as_stream(stream)) != cudaSuccess) {
         cudaGetLastError();
@@ -412,11 +424,25 @@ flora_status flora_set_resample_transfer(flora_set* set, const uint64_t* seeds_o
     flora_status st = FLORA_OK;
     for (size_t i = 0; i < set->S.size() && st == FLORA_OK; ++i) {
         if (set->S[i].rows == 0) continue;
-        st = transfer_with_scratch(&set->S[i], &set->S[i], big[i].cols, big[i].dtype, seeds_old[i], seeds_new[i], 1.0f,
+        st = transfer_with_scratch(&set->S[i], &set->S[i], big[i].cols, big[i].dtype, seeds_old[i], seeds_new[i], a,
                                    0.0f, T, as_stream(stream));
     }
     if (cudaFreeAsync(T, as_stream(stream)) != cudaSuccess && st == FLORA_OK) st = FLORA_ERR_CUDA;
     return st;
+}
+
+flora_status flora_set_resample_transfer(flora_set* set, const uint64_t* seeds_old, const uint64_t* seeds_new, void* stream)
+{
+    return set_transfer(set, seeds_old, seeds_new, 1.0f, stream);
+}
+
+flora_status flora_set_momentum_step_resampled(flora_set* set, float beta, const uint64_t* seeds_old, const uint64_t* seeds_new, void* stream)
+{
+    if (!set || !seeds_old || !seeds_new) return FLORA_ERR_NULL;
+    if (!set->has_G) return FLORA_ERR_UNSUPPORTED;
+    flora_status st = set_transfer(set, seeds_old, seeds_new, beta, stream);
+    if (st) return st;
+    return set_compress(set, seeds_new, 1.0f - beta, 1.0f, stream);
 }
 
 flora_status flora_set_zero_state(flora_set* set, void* stream)

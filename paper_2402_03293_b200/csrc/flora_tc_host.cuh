@@ -508,7 +508,7 @@ inline flora_status tc_set_build_on(TcSet& set, const std::vector<flora_mat>& G,
     set.r = (int)S[0].cols;
     bool g_ok = !G.empty(), w_ok = !W.empty();
     for (size_t i = 0; i < S.size(); ++i) {
-        if (!G.empty() && !tc_mat_ok(G[i])) g_ok = false;
+        if (!G.empty() && (!tc_mat_ok(G[i]) || !tc_sketch_ok(S[i]))) g_ok = false;       // the epilogue writes S through its tensor map
         if (!W.empty() && (!tc_mat_ok(W[i]) || !tc_sketch_ok(S[i]))) w_ok = false;
     }
     if (!g_ok && !w_ok) return FLORA_OK;

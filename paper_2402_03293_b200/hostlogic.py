@@ -47,22 +47,30 @@ class MomentumState:
     """Algorithm 2: at steps t = 0 mod kappa the projection is resampled and M is carried over by
     M <- M A_old A_new^T; then M <- beta M + (1-beta) G A_new^T and the update M A_new is applied."""
 
-    def __init__(self, ops, count: int, beta: float, kappa: int, base_seed: int = 0, skip_transfer_of_zero_state: bool = True):
+    def __init__(self, ops, count: int, beta: float, kappa: int, base_seed: int = 0, skip_transfer_of_zero_state: bool = True,
+                 fuse_transfer: bool = True):
         self.ops, self.count, self.beta, self.kappa, self.base_seed = ops, count, beta, kappa, base_seed
         self.t = 0
         self.epoch = 0
         self.skip0 = skip_transfer_of_zero_state
+        self.fuse = fuse_transfer                        # transfer and update of a resampling step as one call
 
     def seeds(self, epoch: int) -> List[int]:
         return [binding.flora_derive_seed(self.base_seed, i, epoch) for i in range(self.count)]
 
     def step(self, lr: float, stream=None) -> None:
+        fused = False
         if binding.flora_resamples_at(self.t, self.kappa):
             old, new = self.seeds(self.epoch), self.seeds(self.epoch + 1)
             if not (self.t == 0 and self.skip0):          # M = 0 at t = 0: the transfer of zeros is zeros
-                self.ops.resample_transfer(old, new, stream)
+                if self.fuse:
+                    self.ops.momentum_step_resampled(self.beta, old, new, stream)   # transfer and update in one call
+                    fused = True
+                else:
+                    self.ops.resample_transfer(old, new, stream)
             self.epoch += 1
         cur = self.seeds(self.epoch)
-        self.ops.momentum_step(self.beta, cur, stream)
+        if not fused:
+            self.ops.momentum_step(self.beta, cur, stream)
         self.ops.decompress_apply(cur, lr, 1.0, stream)
         self.t += 1

@@ -3,7 +3,8 @@
     python -m paper_2402_03293_b200.measure gpt2_xl_set
     python -m paper_2402_03293_b200.measure single_bf16_4096x11008 --rank 128 --ops compress decompress
 
-Each operation (compress-accumulate, momentum step, decompress-apply, resample transfer) runs over the whole
+Each operation (compress-accumulate, momentum step, decompress-apply, resample transfer, and the resampling
+momentum step that combines the last two) runs over the whole
 weight set of the workload, back to back, with the inputs resident in device memory; the time is taken with
 CUDA events around `--iters` launches after three warm-up launches.  Gradient sets rotate so that a launch
 never finds its input in L2.  One JSON line per run: microseconds per launch and algorithmic GB/s
@@ -21,7 +22,7 @@ import torch
 from . import binding as fb
 from . import workloads as wl
 
-OPS = ("compress", "momentum", "decompress", "transfer")
+OPS = ("compress", "momentum", "decompress", "transfer", "momentum_resampled")
 
 
 def main() -> None:
@@ -74,6 +75,9 @@ def main() -> None:
     if "transfer" in args.ops:
         t = timed(lambda i: sets[0].resample_transfer(seeds, new_seeds), max(1, args.iters // 4))
         out["transfer_us"] = round(t, 1)
+    if "momentum_resampled" in args.ops:
+        t = timed(lambda i: sets[i % n_sets].momentum_step_resampled(0.9, seeds, new_seeds), max(1, args.iters // 4))
+        out["momentum_resampled_us"] = round(t, 1)
     for s in sets:
         s.close()
     if fb.flora_device_status() != 0:

@@ -74,6 +74,12 @@ class _Mirror:
         for i, rp in self.replays.items():
             rp.transfer(old[i], new[i])
 
+    def momentum_step_resampled(self, beta, old, new, stream=None):
+        self.fset.momentum_step_resampled(beta, old, new, stream)
+        for i, rp in self.replays.items():                        # the oracle takes Algorithm 2's two steps in order
+            rp.transfer(old[i], new[i])
+            rp.momentum(self.G()[i], beta, new[i])
+
     def decompress_apply(self, seeds, lr, scale, stream=None):
         self.fset.decompress_apply(seeds, lr, scale, stream)
         for i, rp in self.replays.items():

@@ -345,3 +345,29 @@ def test_repeated_launches_are_bit_identical(n, m, r):
             else:
                 assert rel_err(C.cpu().numpy(), first_c.cpu().numpy()) <= 1e-5
     assert fb.flora_device_status() == 0
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("n,m,r", [(9, 33, 4), (300, 1024, 32), (256, 4096, 128), (1000, 515, 17)])
+def test_resampled_momentum_step(n, m, r, dtype):
+    """Algorithm 2 at a resampling step as one call, against the oracle's transfer followed by its momentum step."""
+    G = _g(n, m, dtype, 21)
+    M0 = torch.randn(n, r, device=DEV)
+    M = M0.clone()
+    fb.flora_momentum_step_resampled(G, M, 0.9, 40, 41)
+    ref = wl.as_numpy(M0).copy()
+    orc.momentum_step_resampled(wl.as_numpy(G), orc.projection(40, r, m, dtype), orc.projection(41, r, m, dtype), 0.9, ref)
+    assert rel_err(M.cpu().numpy(), ref) <= TOL[dtype]
+    # and the set-level call over several matrices
+    shapes = [(256, 512), (384, 1024), (128, 64)]
+    Gs = [_g(a, b, "bf16", 30 + i) for i, (a, b) in enumerate(shapes)]
+    Ms = [torch.randn(a, r, device=DEV) for a, _ in shapes]
+    M0s = [x.clone() for x in Ms]
+    fset = fb.FloraSet(Gs, None, Ms)
+    old, new = [50, 51, 52], [60, 61, 62]
+    fset.momentum_step_resampled(0.5, old, new)
+    for i, (a, b) in enumerate(shapes):
+        ref = wl.as_numpy(M0s[i]).copy()
+        orc.momentum_step_resampled(wl.as_numpy(Gs[i]), orc.projection(old[i], r, b, "bf16"), orc.projection(new[i], r, b, "bf16"), 0.5, ref)
+        assert rel_err(Ms[i].cpu().numpy(), ref) <= TOL["bf16"], i
+    fset.close()

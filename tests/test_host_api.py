@@ -116,7 +116,7 @@ def test_accumulation_cycle_order_algorithm_1():
 
 def test_momentum_order_algorithm_2():
     ops = _Recorder()
-    mom = hostlogic.MomentumState(ops, count=2, beta=0.9, kappa=3, base_seed=5)
+    mom = hostlogic.MomentumState(ops, count=2, beta=0.9, kappa=3, base_seed=5, fuse_transfer=False)
     for _ in range(7):
         mom.step(0.1)
     names = [c[0] for c in ops.calls]
@@ -128,6 +128,14 @@ def test_momentum_order_algorithm_2():
     assert tr[1] == ops.calls[4][2] and tr[2] == ops.calls[7][2] == ops.calls[8][1]
     assert ops.calls[0][1] == 0.9 and ops.calls[1][2:] == (0.1, 1.0)
     ops2 = _Recorder()
-    mom2 = hostlogic.MomentumState(ops2, count=1, beta=0.5, kappa=1, skip_transfer_of_zero_state=False)
+    mom2 = hostlogic.MomentumState(ops2, count=1, beta=0.5, kappa=1, skip_transfer_of_zero_state=False, fuse_transfer=False)
     mom2.step(1.0)
     assert [c[0] for c in ops2.calls] == ["resample_transfer", "momentum_step", "decompress_apply"]
+    # by default a resampling step is one call that carries both seed lists
+    ops3 = _Recorder()
+    mom3 = hostlogic.MomentumState(ops3, count=2, beta=0.9, kappa=3, base_seed=5)
+    for _ in range(4):
+        mom3.step(0.1)
+    assert [c[0] for c in ops3.calls] == ["momentum_step", "decompress_apply"] * 3 + ["momentum_step_resampled", "decompress_apply"]
+    fused = ops3.calls[6]
+    assert fused[1] == 0.9 and fused[2] == ops3.calls[4][2] and fused[3] == ops3.calls[7][1]

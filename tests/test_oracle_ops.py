@@ -308,3 +308,28 @@ def test_state_is_a_fraction_r_over_m_of_the_matrix():
     w = wl.WORKLOADS["gpt2_small_set"]
     state = sum(n * w.r for n, _ in w.shapes)
     assert state * 4 == 8257536 and w.elements == 84934656
+
+
+def test_resampled_momentum_step_is_the_closed_form_of_algorithm_2():
+    """beta (M A_old A_new^T) + (1 - beta) G A_new^T with materialised projections, in float64."""
+    n, m, r, beta = 5, 21, 4, 0.8
+    rng = _rng(12)
+    G = rng.standard_normal((n, m)).astype(np.float32)
+    M0 = rng.standard_normal((n, r)).astype(np.float32)
+    Ao, An = orc.materialize_A(300, r, m), orc.materialize_A(301, r, m)
+    M = M0.copy()
+    orc.momentum_step_resampled(G, Ao, An, beta, M)
+    g, m0, ao, an = (x.astype(np.float64) for x in (G, M0, Ao, An))
+    ref = beta * (m0 @ ao @ an.T) + (1.0 - beta) * (g @ an.T)
+    assert np.allclose(M, ref, rtol=2e-6, atol=2e-6)
+    # the two special cases: beta = 1 is the transfer alone, beta = 0 forgets the old state altogether
+    M = M0.copy()
+    orc.momentum_step_resampled(G, Ao, An, 1.0, M)
+    T = M0.copy()
+    orc.resample_transfer(T, Ao, An)
+    assert np.array_equal(M, T)
+    M = M0.copy()
+    orc.momentum_step_resampled(G, Ao, An, 0.0, M)
+    C = np.zeros_like(M0)
+    orc.compress_accumulate(G, An, C)
+    assert np.array_equal(M, C)
