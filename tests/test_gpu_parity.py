@@ -371,3 +371,46 @@ def test_resampled_momentum_step(n, m, r, dtype):
         orc.momentum_step_resampled(wl.as_numpy(Gs[i]), orc.projection(old[i], r, b, "bf16"), orc.projection(new[i], r, b, "bf16"), 0.5, ref)
         assert rel_err(Ms[i].cpu().numpy(), ref) <= TOL["bf16"], i
     fset.close()
+
+
+@pytest.mark.parametrize("case", range(14))
+def test_random_sets_against_oracle(case):
+    """Seeded random weight sets (shapes on both sides of every eligibility rule of the tensor-core path, ranks that are
+    and are not multiples of 4, 16, 64), run through every set-level operation and compared with the oracle."""
+    rng = np.random.default_rng(1000 + case)
+    r = int(rng.choice([1, 4, 8, 17, 32, 48, 64, 100, 128, 200, 256]))
+    count = int(rng.integers(1, 5))
+    eligible = case % 3 != 0                     # two thirds of the cases: every matrix large and aligned enough for tcgen05
+    shapes = []
+    for _ in range(count):
+        if eligible:
+            shapes.append((int(rng.integers(128, 700)), int(rng.integers(8, 300)) * 8))
+        else:
+            shapes.append((int(rng.integers(1, 300)), int(rng.integers(1, 700))))
+    G = [_g(n, m, "bf16", 100 * case + i) for i, (n, m) in enumerate(shapes)]
+    W = [(torch.randn(n, m, device=DEV) * 0.02).to(torch.bfloat16) for n, m in shapes]
+    W0 = [x.clone() for x in W]
+    S = [torch.zeros(n, r, device=DEV) for n, _ in shapes]
+    fset = fb.FloraSet(G, W, S)
+    s0 = [int(x) for x in rng.integers(1, 2 ** 62, size=count)]
+    s1 = [int(x) for x in rng.integers(1, 2 ** 62, size=count)]
+    fset.compress_accumulate(s0)
+    fset.compress_accumulate(s0)
+    fset.momentum_step(0.7, s0)
+    fset.momentum_step_resampled(0.6, s0, s1)
+    fset.decompress_apply(s1, 0.5, 0.25)
+    torch.cuda.synchronize()
+    assert fb.flora_device_status() == 0
+    for i, (n, m) in enumerate(shapes):
+        A0, A1 = orc.projection(s0[i], r, m, "bf16"), orc.projection(s1[i], r, m, "bf16")
+        g = wl.as_numpy(G[i])
+        ref = np.zeros((n, r), dtype=np.float32)
+        orc.compress_accumulate(g, A0, ref)
+        orc.compress_accumulate(g, A0, ref)
+        orc.momentum_step(g, A0, 0.7, ref)
+        orc.momentum_step_resampled(g, A0, A1, 0.6, ref)
+        assert rel_err(S[i].cpu().numpy(), ref) <= TOL["bf16"], (case, i, "sketch")
+        w = wl.as_numpy(W0[i]).copy()
+        orc.decompress_apply(w, S[i].cpu().numpy(), A1, 0.5, 0.25)
+        assert rel_err(values(wl.as_numpy(W[i])), values(w)) <= TOL["bf16"], (case, i, "weights")
+    fset.close()
