@@ -105,8 +105,8 @@ def test_transfer(n, m, r, operand):
     assert rel_err(dst.cpu().numpy(), oracle_transfer(M0, src, m, operand, 3, 4, 0.0125, 0.9)) <= TOL[operand]
 
 
-def test_strided_views_are_honoured():
-    n, m, r = 70, 200, 16
+@pytest.mark.parametrize("n,m,r", [(70, 200, 16), (300, 1000, 20), (384, 2048, 200)])     # SIMT path; tensor-core paths with ragged tiles
+def test_strided_views_are_honoured(n, m, r):
     Gbig = _g(n, m + 24, "bf16", 3)
     Cbig = torch.zeros(n, r + 8, device=DEV)
     fb.flora_compress_accumulate(Gbig[:, :m], Cbig[:, :r], 9, r)
@@ -119,6 +119,14 @@ def test_strided_views_are_honoured():
     refw = oracle_decompress(W0[:, :m].contiguous(), Cbig[:, :r].contiguous(), 9, 1.0, 1.0)
     assert rel_err(values(wl.as_numpy(Wbig[:, :m].contiguous())), values(refw)) <= TOL["bf16"]
     assert torch.equal(Wbig[:, m:], W0[:, m:])
+    # momentum (read-modify-write of the strided sketch) and the transfer leave the columns beside the view alone
+    Mbig = torch.randn(n, r + 8, device=DEV)
+    M0 = Mbig.clone()
+    fb.flora_momentum_step(Gbig[:, :m], Mbig[:, :r], 0.9, 9)
+    ref = oracle_compress(Gbig[:, :m].contiguous(), M0[:, :r].contiguous(), 9, a=0.1, b=0.9)
+    assert rel_err(Mbig[:, :r].cpu().numpy(), ref) <= TOL["bf16"]
+    fb.flora_resample_transfer(Mbig[:, :r], m, "bf16", 9, 10)
+    assert torch.equal(Mbig[:, r:], M0[:, r:])
 
 
 def test_empty_inputs():
