@@ -204,13 +204,14 @@ def flora_debug_force_path(path: int) -> None:
 def flora_debug_plan(shapes, r: int, which: str):
     """Work items and launch parameters the library would use for bf16 matrices of these (rows, cols) shapes.
 
-    which = "compress" or "decompress".  Returns (items, params): items as a list of tuples, params as a tuple of
+    which = "compress", "decompress" or "compress_slots" (the per-cluster unit lists of the persistent compression
+    kernel that serves ranks above 64).  Returns (items, params): items as a list of tuples, params as a tuple of
     eight ints (see include/flora.h).  No kernel runs; usable without a GPU."""
     count = len(shapes)
     rows = (ctypes.c_int64 * max(count, 1))(*[int(n) for n, _ in shapes])
     cols = (ctypes.c_int64 * max(count, 1))(*[int(m) for _, m in shapes])
-    w = 0 if which == "compress" else 1
-    width = 6 if w == 0 else 4
+    w = {"compress": 0, "decompress": 1, "compress_slots": 2}[which]
+    width = {0: 6, 1: 4, 2: 1}[w]
     n = ctypes.c_int64(0)
     params = (ctypes.c_int32 * 8)()
     _check(load().flora_debug_plan(rows, cols, count, r, w, None, 0, ctypes.byref(n), params), "flora_debug_plan")

@@ -522,8 +522,16 @@ flora_status flora_debug_plan(const int64_t* rows, const int64_t* cols, int64_t 
     TcSet set;
     set.count = (int)count;
     set.r = r;
-    const int width = which == 0 ? 6 : 4;
-    if (which == 0) {
+    const int width = which == 0 ? 6 : which == 2 ? 1 : 4;
+    if (which == 2) {
+        // the slot table of the persistent compression kernel (ranks above 64): per launch, one first-unit index per
+        // slot and the unit count; empty for the ranks that run one CTA per item
+        plan_compress(set, mats, r);
+        *n_items = (int64_t)set.h_slots.size();
+        const int32_t p[8] = {set.T, set.S, set.gstages, set.astages, set.GW, set.P, (int32_t)(set.k1_launch_begin.size() - 1), (int32_t)set.k1_smem};
+        memcpy(params, p, sizeof(p));
+        for (int64_t i = 0; i < std::min<int64_t>(*n_items, capacity); ++i) items[i] = set.h_slots[(size_t)i];
+    } else if (which == 0) {
         plan_compress(set, mats, r);
         *n_items = (int64_t)set.h_k1.size();
         const int32_t p[8] = {set.T, set.S, set.gstages, set.astages, set.GW, set.P, (int32_t)(set.k1_launch_begin.size() - 1), (int32_t)set.k1_smem};

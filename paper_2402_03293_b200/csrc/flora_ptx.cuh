@@ -224,6 +224,22 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 
+// The same for a CTA pair (cta_group::2): one warp of each of the two CTAs executes; both tensor memories get the
+// same columns, and MMAs issued for the pair write the accumulator rows 0..127 into the even CTA's tensor memory and
+// rows 128..255 into the odd CTA's.
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
 // Shared-memory operand descriptor, K-major, 128-byte swizzle: rows of 128 bytes, groups of eight
 // rows 1024 bytes apart.  `addr` is the shared address of the first row (+ the byte offset of the
 // current 16-element K slice inside the 128-byte row); the tile base is 1024-byte aligned.
@@ -276,6 +292,31 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
 __device__ __forceinline__ void umma_commit_cluster(uint32_t bar, uint16_t cta_mask)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(cta_mask)
+                 : "memory");
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = m (128, or 256 for a CTA pair), N = n.
+__device__ __forceinline__ uint32_t umma_idesc_bf16_mn(uint32_t m, uint32_t n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((m >> 4) << 24);
+}
+// MMA of a CTA pair, issued by one thread of the even CTA: D (256 x N, rows split over the two tensor memories)
+// (+)= A (256 x 16, each CTA's 128 rows from its own shared memory) * B^T (N x 16, each CTA holds N/2 rows).
+// The descriptors name shared-memory offsets that are valid in both CTAs.
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrives on the mbarrier at this shared-memory offset in every CTA of `cta_mask` once every MMA issued so far for
+// the pair has completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t cta_mask)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                  ::"r"(bar), "h"(cta_mask)
                  : "memory");
 }

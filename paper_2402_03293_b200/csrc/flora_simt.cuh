@@ -233,13 +233,4 @@ simt_apply_gram_kernel(float* dst, int64_t ldd, const float* src, int64_t lds,
     }
 }
 
-// S <- b S  (pre-scaling of a sketch whose update is split over several blocks)
-__global__ void scale_rows_kernel(float* __restrict__ S, int64_t n, int r, int64_t lds, float b)
-{
-    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= n * r) return;
-    float* p = S + (t / r) * lds + (t % r);
-    *p = (b == 0.0f) ? 0.0f : *p * b;
-}
-
 }  // namespace flora

@@ -11,6 +11,9 @@
 #include <atomic>
 #include <vector>
 
+#include <mutex>
+
+#include "flora_pair.cuh"
 #include "flora_pool.cuh"
 #include "flora_tc.cuh"
 
@@ -34,6 +37,12 @@ struct TcSet {
     std::vector<K1Item> h_k1;
     std::vector<int> k1_launch_begin;   // item ranges per launch (at most SEEDS_PER_LAUNCH matrices each)
     std::vector<int> split_mats;        // matrices whose sketch is updated by several items
+    // ranks above 64: the persistent CTA-pair kernel; a launch's clusters ("slots") each walk their own list of units
+    bool k1_pair = false;
+    int k1_n = 0;                       // accumulator columns: r rounded up to a multiple of 64
+    std::vector<int> h_slots;           // per launch: slots + 1 first-unit indices (relative to the launch's first unit)
+    std::vector<int> k1_slots_begin;    // where each launch's table starts in h_slots
+    int* d_slots = nullptr;
     // decompression
     int bn = 128, slots = 2, cstages = 2, k2_gw = 8, k2_nslabs = 2, k2_grid_max = 148;
     bool k2_bf16 = false;               // ranks above 64: the kernel reads a bf16 copy of the sketches
@@ -118,13 +127,235 @@ inline int sm_count()
 
 constexpr size_t SMEM_BUDGET = 226 * 1024;   // per SM, below the 227 KB limit of sm_100
 
-// Tuning knobs (environment variables, read when a set is planned): they change tile shapes and the
-// work split only, never what is computed.
+// Tile shapes and the work split are chosen by the planners below.  A build with -DFLORA_TUNE lets environment
+// variables override single choices for parameter sweeps (they never change what is computed); the library as
+// shipped reads no environment variable.
+#ifdef FLORA_TUNE
 inline int tune_knob(const char* name, int dflt, int lo, int hi)
 {
     const char* v = getenv(name);
     if (!v || !*v) return dflt;
     return std::max(lo, std::min(hi, atoi(v)));
+}
+#else
+inline int tune_knob(const char*, int dflt, int, int) { return dflt; }
+#endif
+
+// Lifts a kernel's limit on dynamic shared memory to what the device allows, once per kernel and device.  The
+// attribute belongs to the function, not to a launch: it is raised to the maximum once and never lowered, so sets
+// with different footprints can be alive, and launched in any order, at the same time.
+template <auto Kernel>
+inline bool raise_smem_limit()
+{
+    static std::mutex mutex;
+    static bool done[POOL_MAX_DEVICES] = {};
+    int dev = -1, optin = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= POOL_MAX_DEVICES) {
+        cudaGetLastError();
+        return false;
+    }
+    std::lock_guard<std::mutex> lock(mutex);
+    if (done[dev]) return true;
+    if (cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
+        cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    done[dev] = true;
+    return true;
+}
+
+// Clusters of `S` CTAs of `Kernel` that can be resident at once (fewer than SMs / S: a cluster sits inside one GPC);
+// SMs / S when there is no device to ask.
+template <auto Kernel>
+inline int resident_clusters(int S, int threads, size_t smem)
+{
+    int slots = std::max(1, sm_count() / S);
+    if (!raise_smem_limit<Kernel>()) return slots;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(S * 64));
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int active = 0;
+    if (cudaOccupancyMaxActiveClusters(&active, Kernel, &cfg) == cudaSuccess && active > 0) slots = active;
+    else cudaGetLastError();
+    return slots;
+}
+
+// Cost model of the compression planners, in units of one 64-column step of a full CTA: what a work unit costs
+// before its first and after its last step (barriers, first loads, writing the accumulators out).
+constexpr double K1_UNIT_OVERHEAD_STEPS = 6.0;
+// Values of A that the generator warps of one SM produce while the SM streams one 64-column step of two G tiles
+// (about 0.6 us): the cluster is made large enough that a CTA's share of a tile stays below this.
+constexpr int PAIR_VALUES_PER_STEP = 2048;
+
+// Work decomposition of compress_pair_kernel (ranks above 64).
+//
+// A unit is (matrix, group of up to S * PAIR_T 128-row tiles, range of 64-column steps); a cluster of S CTAs
+// (S/2 pairs) handles one unit at a time, the CTAs taking consecutive rows.  Units are balanced over the clusters
+// that can be resident ("slots"), largest first; every slot gets its own list, which its cluster walks.
+inline void plan_compress_pair(TcSet& set, const std::vector<flora_mat>& G, int r)
+{
+    const int N = (r + 63) & ~63;
+    const int T = PAIR_T;
+    int64_t max_tiles = 1, total_work = 0;
+    for (const auto& g : G) {
+        const int64_t tiles = (g.rows + 127) / 128, ks = (g.cols + 63) / 64;
+        max_tiles = std::max(max_tiles, tiles);
+        total_work += tiles * ks;
+    }
+    int S = 2;
+    while (S < 8 && N * 64 / S > PAIR_VALUES_PER_STEP) S <<= 1;
+    while (S > 2 && (int64_t)S * T > 2 * max_tiles) S >>= 1;          // not more CTAs than there are rows to share
+    S = tune_knob("FLORA_K1_CLUSTER", S, 2, 8);
+    if (S & (S - 1)) S = 2;
+    const size_t g_stage = (size_t)T * G_TILE_BYTES, a_stage = (size_t)(N / 2) * 128, staging = 2 * (size_t)S_CHUNK_BYTES_K1;
+    const size_t ring_budget = SMEM_BUDGET - sizeof(PairSmem) - 1024 - staging;
+    // A tiles are made on chip and travel between the CTAs of a cluster, whose slowest member paces all: four stages
+    // (three when that leaves fewer than three for G).  The G tiles come from HBM and get the rest.
+    int astages = 4;
+    if ((ring_budget - astages * a_stage) / g_stage < 3) astages = 3;
+    astages = tune_knob("FLORA_K1_ASTAGES", astages, 2, 8);
+    int gstages = (int)std::min<size_t>(PAIR_RELAY_DEPTH - 1, (ring_budget - astages * a_stage) / g_stage);
+    gstages = tune_knob("FLORA_K1_GSTAGES", std::max(1, gstages), 1, std::max(1, gstages));
+    int GW = tune_knob("FLORA_K1_GEN_WARPS", PAIR_MAX_GEN_WARPS, 4, PAIR_MAX_GEN_WARPS) & ~3;
+    // generator teams: as many as keep every thread of a team busy with at least one task per slice
+    {
+        const int tile_tasks = N / S * 8;
+        int P = 1;
+        while (2 * P <= astages && GW % (2 * P) == 0 && 32 * GW / (2 * P) >= tile_tasks) P *= 2;
+        P = tune_knob("FLORA_K1_TEAMS", P, 1, 8);
+        while (P > 1 && (GW % P || P > astages || (P & (P - 1)))) --P;
+        set.P = P;
+    }
+    set.k1_pair = true;
+    set.k1_n = N;
+    set.T = T;
+    set.S = S;
+    set.GW = GW;
+    set.gstages = gstages;
+    set.astages = astages;
+    set.k1_smem = (size_t)gstages * g_stage + (size_t)astages * a_stage + staging + sizeof(PairSmem) + 1024;
+    const int64_t slots = resident_clusters<compress_pair_kernel>(S, pair_threads(GW), set.k1_smem);
+    const int64_t group_tiles = (int64_t)S * T;
+    struct Unit { int mat; int64_t tile0, tiles, kstep0, ksteps; bool direct; };
+    auto build_units = [&](int64_t target, std::vector<Unit>& units, std::vector<int>& split) {
+        units.clear();
+        split.clear();
+        for (size_t i = 0; i < G.size(); ++i) {
+            const auto& g = G[i];
+            if (g.rows == 0 || g.cols == 0) continue;
+            const int64_t tiles = (g.rows + 127) / 128, ks = (g.cols + 63) / 64;
+            const int64_t groups = (tiles + group_tiles - 1) / group_tiles;
+            const int64_t per_group = (tiles + groups - 1) / groups;     // rows spread evenly over the groups
+            int64_t chunk = std::max<int64_t>(8, target / per_group);
+            int64_t nchunks = (ks + chunk - 1) / chunk;
+            if (nchunks > 1 && ks - (nchunks - 1) * chunk < chunk / 2) --nchunks;    // no short tail unit
+            chunk = (ks + nchunks - 1) / nchunks;
+            nchunks = (ks + chunk - 1) / chunk;
+            if (nchunks > 1) split.push_back((int)i);
+            for (int64_t t0 = 0; t0 < tiles; t0 += per_group)
+                for (int64_t c = 0; c < nchunks; ++c)
+                    units.push_back({(int)i, t0, std::min(per_group, tiles - t0), c * chunk, std::min(chunk, ks - c * chunk), nchunks == 1});
+        }
+    };
+    // a cluster moves in lockstep and every step costs a full CTA's worth of MMAs: a unit's time is its steps plus
+    // the fixed cost of starting and finishing it
+    auto unit_time = [&](const Unit& u) { return K1_UNIT_OVERHEAD_STEPS + (double)u.ksteps; };
+    // longest-processing-time assignment of units[first, last) to the slots; returns the makespan
+    auto assign = [&](const std::vector<Unit>& units, size_t first, size_t last, std::vector<std::vector<int>>* lists) {
+        std::vector<int> order;
+        for (size_t u = first; u < last; ++u) order.push_back((int)u);
+        std::stable_sort(order.begin(), order.end(), [&](int x, int y) { return unit_time(units[x]) > unit_time(units[y]); });
+        std::vector<std::pair<double, int>> heap;                // (time assigned, slot), smallest time on top
+        for (int s = 0; s < (int)slots; ++s) heap.push_back({0.0, s});
+        auto cmp = [](const std::pair<double, int>& x, const std::pair<double, int>& y) { return x.first > y.first || (x.first == y.first && x.second > y.second); };
+        std::make_heap(heap.begin(), heap.end(), cmp);
+        if (lists) lists->assign((size_t)slots, std::vector<int>());
+        double span = 0.0;
+        for (int u : order) {
+            std::pop_heap(heap.begin(), heap.end(), cmp);
+            heap.back().first += unit_time(units[u]);
+            span = std::max(span, heap.back().first);
+            if (lists) (*lists)[(size_t)heap.back().second].push_back(u);
+            std::push_heap(heap.begin(), heap.end(), cmp);
+        }
+        return span;
+    };
+    // column chunks: try several granularities (about 1..4 units per slot) and keep the shortest schedule
+    std::vector<Unit> units, cand_units;
+    std::vector<int> cand_split;
+    double best_span = 1e300;
+    for (int w = 1; w <= 4; ++w) {
+        for (double f : {1.0, 1.1, 1.2, 1.35, 1.5}) {
+            const int64_t target = (int64_t)((double)total_work / (double)(w * slots * group_tiles) * f * (double)group_tiles) + 1;
+            build_units(target, cand_units, cand_split);
+            const double span = assign(cand_units, 0, cand_units.size(), nullptr);
+            if (span < best_span * 0.98) {
+                best_span = span;
+                units = cand_units;
+                set.split_mats = cand_split;
+            }
+        }
+    }
+    // a schedule without any split over columns is preferred when it is nearly as short: every row of a sketch then
+    // has one owner, so a momentum update needs neither the pre-scaling pass nor atomic adds
+    build_units((int64_t)1 << 60, cand_units, cand_split);
+    if (assign(cand_units, 0, cand_units.size(), nullptr) <= 1.12 * best_span) {
+        units = cand_units;
+        set.split_mats = cand_split;
+    }
+    // launches cover at most SEEDS_PER_LAUNCH consecutive matrices (units are in matrix order)
+    set.h_k1.clear();
+    set.h_slots.clear();
+    set.k1_launch_begin.clear();
+    set.k1_launch_first_mat.clear();
+    set.k1_slots_begin.clear();
+    size_t u0 = 0;
+    while (u0 < units.size()) {
+        size_t u1 = u0;
+        while (u1 < units.size() && units[u1].mat < units[u0].mat + SEEDS_PER_LAUNCH) ++u1;
+        std::vector<std::vector<int>> lists;
+        assign(units, u0, u1, &lists);
+        set.k1_launch_begin.push_back((int)set.h_k1.size());
+        set.k1_launch_first_mat.push_back(units[u0].mat);
+        set.k1_slots_begin.push_back((int)set.h_slots.size());
+        int emitted = 0;                                        // units of this launch so far
+        for (const auto& list : lists) {
+            if (list.empty()) continue;                         // slots without work are not launched
+            set.h_slots.push_back(emitted);
+            for (int u : list) {
+                // the unit's tiles spread evenly over the S CTAs of the cluster (some may get none)
+                const Unit& un = units[(size_t)u];
+                int64_t t0 = un.tile0;
+                for (int c = 0; c < S; ++c) {
+                    const int64_t left = un.tile0 + un.tiles - t0;
+                    const int64_t mine = std::min<int64_t>(T, (left + (S - c) - 1) / (S - c));
+                    K1Item it;
+                    it.mat = un.mat;
+                    it.row0 = (int)(t0 * 128);
+                    it.tiles = (int)std::max<int64_t>(0, mine);
+                    it.kstep0 = (int)un.kstep0;
+                    it.ksteps = (int)un.ksteps;
+                    it.direct = un.direct;
+                    set.h_k1.push_back(it);
+                    t0 += it.tiles;
+                }
+                ++emitted;
+            }
+        }
+        set.h_slots.push_back(emitted);
+        u0 = u1;
+    }
+    set.k1_launch_begin.push_back((int)set.h_k1.size());
+    set.k1_slots_begin.push_back((int)set.h_slots.size());
 }
 
 // Work decomposition of the compression kernel over a set of matrices.
@@ -135,6 +366,11 @@ inline int tune_knob(const char* name, int dflt, int lo, int hi)
 // so that the former stays under half of the latter.
 inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
 {
+    if (r > 64) {
+        plan_compress_pair(set, G, r);
+        return;
+    }
+    set.k1_pair = false;
     const int r_pad = (r + 15) & ~15;
     int64_t max_tiles = 1, total_work = 0;       // work unit: one 128-row tile over one 64-column step
     for (const auto& g : G) {
@@ -205,25 +441,7 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
     set.k1_smem = (size_t)gstages * g_stage + (size_t)astages * a_stage + sizeof(K1Smem) + 1024;
     // column chunks: aim at about `waves` items per slot (a slot is a CTA, or a cluster), at least 8 steps each
     int64_t slots = std::max<int64_t>(1, (int64_t)sm_count() * per_sm / S);
-    if (cudaFuncSetAttribute(compress_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)set.k1_smem) != cudaSuccess) cudaGetLastError();
-    if (S > 1) {
-        // clusters that can be resident at once (fewer than SMs / S: a cluster must sit inside one GPC)
-        cudaFuncSetAttribute(compress_tc_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 0);
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(S * 64));
-        cfg.blockDim = dim3((unsigned)k1_threads(set.GW));
-        cfg.dynamicSmemBytes = set.k1_smem;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = (unsigned)S;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        int active = 0;
-        if (cudaOccupancyMaxActiveClusters(&active, compress_tc_kernel, &cfg) == cudaSuccess && active > 0) slots = active;
-        else cudaGetLastError();
-    }
+    if (S > 1) slots = resident_clusters<compress_tc_kernel>(S, k1_threads(set.GW), set.k1_smem);
     const int64_t group_tiles = (int64_t)S * T;                      // rows of one slot, in tiles
     struct Unit { int mat; int64_t tile0, tiles, kstep0, ksteps; bool direct; };
     auto build_units = [&](int64_t target, std::vector<Unit>& units, std::vector<int>& split) {
@@ -250,7 +468,7 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
     // scaled by the rows a CTA streams (a cluster moves in lockstep, so its most loaded CTA counts)
     auto unit_time = [&](const Unit& u) {
         const double per_cta = (double)((u.tiles + S - 1) / S);
-        return (6.0 + (double)u.ksteps) * std::max(per_cta, 0.5 * T);
+        return (K1_UNIT_OVERHEAD_STEPS + (double)u.ksteps) * std::max(per_cta, 0.5 * T);
     };
     auto makespan = [&](const std::vector<Unit>& units) {
         std::vector<double> tms;
@@ -445,18 +663,21 @@ inline void tc_set_free_stream(TcSet& s, cudaStream_t st)
         if (s.d_k1) cudaFreeAsync(s.d_k1, st);
         if (s.d_k2) cudaFreeAsync(s.d_k2, st);
         if (s.d_split) cudaFreeAsync(s.d_split, st);
+        if (s.d_slots) cudaFreeAsync(s.d_slots, st);
         if (s.d_sb) cudaFreeAsync(s.d_sb, st);
     } else {
         if (s.d_mats) cudaFree(s.d_mats);
         if (s.d_k1) cudaFree(s.d_k1);
         if (s.d_k2) cudaFree(s.d_k2);
         if (s.d_split) cudaFree(s.d_split);
+        if (s.d_slots) cudaFree(s.d_slots);
         if (s.d_sb) cudaFree(s.d_sb);
     }
     s.d_mats = nullptr;
     s.d_k1 = nullptr;
     s.d_k2 = nullptr;
     s.d_split = nullptr;
+    s.d_slots = nullptr;
     s.d_sb = nullptr;
     s.compress_ready = s.decompress_ready = false;
 }
@@ -555,16 +776,13 @@ inline flora_status tc_set_build_on(TcSet& set, const std::vector<flora_mat>& G,
         if (rc) return rc;
         rc = upload(&set.d_split, set.split_mats, transient, st);
         if (rc) return rc;
-        if (cudaFuncSetAttribute(compress_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)set.k1_smem) != cudaSuccess)
-            return FLORA_ERR_CUDA;
+        rc = upload(&set.d_slots, set.h_slots, transient, st);
+        if (rc) return rc;
         set.compress_ready = true;
     }
     if (w_ok) {
         rc = upload(&set.d_k2, set.h_k2, transient, st);
         if (rc) return rc;
-        cudaError_t e = set.k2_bf16 ? cudaFuncSetAttribute(decompress_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)set.k2_smem)
-                                    : cudaFuncSetAttribute(decompress_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)set.k2_smem);
-        if (e != cudaSuccess) return FLORA_ERR_CUDA;
         set.decompress_ready = true;
     }
     return FLORA_OK;
@@ -613,15 +831,19 @@ inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, 
             launches.fetch_add(1, std::memory_order_relaxed);
         }
     }
+    const bool pair = set.k1_pair;
+    if (!(pair ? raise_smem_limit<compress_pair_kernel>() : raise_smem_limit<compress_tc_kernel>())) return FLORA_ERR_CUDA;
     for (size_t l = 0; l + 1 < set.k1_launch_begin.size(); ++l) {
         const int begin = set.k1_launch_begin[l], end = set.k1_launch_begin[l + 1];
         if (end == begin) continue;
         const int seed_base = set.k1_launch_first_mat[l];
         SeedTable table;
         for (int i = 0; i < SEEDS_PER_LAUNCH; ++i) table.s[i] = seed_base + i < set.count ? seeds[seed_base + i] : 0;
+        // the pair kernel is persistent: one cluster per slot that has work; the other kernel runs one CTA per item
+        const int n_slots = pair ? set.k1_slots_begin[l + 1] - set.k1_slots_begin[l] - 1 : 0;
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(end - begin));
-        cfg.blockDim = dim3((unsigned)k1_threads(set.GW));
+        cfg.gridDim = dim3((unsigned)(pair ? n_slots * set.S : end - begin));
+        cfg.blockDim = dim3((unsigned)(pair ? pair_threads(set.GW) : k1_threads(set.GW)));
         cfg.dynamicSmemBytes = set.k1_smem;
         cfg.stream = st;
         cudaLaunchAttribute attr[2];
@@ -635,9 +857,17 @@ inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, 
         cfg.numAttrs = set.S > 1 ? 2 : 1;
         const TcMatrix* mats = set.d_mats;
         const K1Item* items = set.d_k1 + begin;
-        if (cudaLaunchKernelEx(&cfg, compress_tc_kernel, mats, items, table, seed_base, r, scale, a, b, set.T, set.gstages, set.astages, set.S, set.GW, set.P, l == 0 ? late_wait : 0) !=
-            cudaSuccess)
-            return FLORA_ERR_CUDA;
+        const int lw = l == 0 ? late_wait : 0;
+        cudaError_t e;
+        if (pair) {
+            const int* slot_table = set.d_slots + set.k1_slots_begin[l];
+            e = cudaLaunchKernelEx(&cfg, compress_pair_kernel, mats, items, slot_table, table, seed_base, r, set.k1_n, scale, a, b, set.gstages,
+                                   set.astages, set.S, set.GW, set.P, lw);
+        } else {
+            e = cudaLaunchKernelEx(&cfg, compress_tc_kernel, mats, items, table, seed_base, r, scale, a, b, set.T, set.gstages, set.astages, set.S,
+                                   set.GW, set.P, lw);
+        }
+        if (e != cudaSuccess) return FLORA_ERR_CUDA;
         launches.fetch_add(1, std::memory_order_relaxed);
     }
     return cudaPeekAtLastError() == cudaSuccess ? FLORA_OK : FLORA_ERR_CUDA;
@@ -670,6 +900,7 @@ inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float s
             launches.fetch_add(1, std::memory_order_relaxed);
         }
     }
+    if (!(set.k2_bf16 ? raise_smem_limit<decompress_tc_kernel<true>>() : raise_smem_limit<decompress_tc_kernel<false>>())) return FLORA_ERR_CUDA;
     for (size_t l = 0; l + 1 < set.k2_launch_begin.size(); ++l) {
         const int begin = set.k2_launch_begin[l], end = set.k2_launch_begin[l + 1];
         if (end == begin) continue;

@@ -33,9 +33,11 @@ def tiles_of(n):
 def test_compression_items_cover_every_tile_and_step_once(name, r):
     shapes = SHAPE_SETS[name]
     items, (T, S, gstages, astages, gen_warps, teams, launches, smem) = fb.flora_debug_plan(shapes, r, "compress")
-    r_pad = (r + 15) // 16 * 16
+    # accumulator columns: r rounded up to 16, or to 64 for the ranks that run on CTA pairs
+    r_pad = (r + 15) // 16 * 16 if r <= 64 else (r + 63) // 64 * 64
     assert 1 <= T and T * r_pad <= 512                         # accumulators fit tensor memory
     assert S in (1, 2, 4, 8) and r_pad % (8 * S) == 0          # portable cluster sizes; whole 8-row groups per CTA
+    assert r <= 64 or S >= 2                                   # pairs
     assert gstages >= 1 and astages >= 1 and smem <= SMEM_LIMIT
     assert 1 <= teams <= astages and gen_warps % teams == 0
     assert launches == (len(shapes) + 447) // 448
@@ -64,6 +66,32 @@ def test_compression_items_cover_every_tile_and_step_once(name, r):
     assert len(seen) == expected and all(v == 1 for v in seen.values())
     for (mat, _, _, k0, ks, direct) in items:                  # an item owns its rows iff the matrix is not cut along the columns
         assert direct == (1 if len(split[mat]) == 1 else 0)
+
+
+@pytest.mark.parametrize("name", sorted(SHAPE_SETS))
+@pytest.mark.parametrize("r", RANKS)
+def test_persistent_compression_slots_partition_the_units(name, r):
+    """Ranks above 64: every launch lists, per cluster slot, a contiguous non-empty range of its units; together the
+    ranges cover the launch's units once, and no launch asks for more clusters than 148 SMs could hold."""
+    shapes = SHAPE_SETS[name]
+    items, (T, S, *_rest, launches, _smem) = fb.flora_debug_plan(shapes, r, "compress")
+    table, _ = fb.flora_debug_plan(shapes, r, "compress_slots")
+    table = [t[0] for t in table]
+    if r <= 64:
+        assert table == []
+        return
+    units_total = len(items) // S
+    covered, pos = 0, 0
+    for _ in range(launches):
+        assert table[pos] == 0
+        end = pos + 1
+        while end < len(table) and table[end] > table[end - 1]:
+            end += 1
+        begins = table[pos:end]
+        assert len(begins) >= 2 and len(begins) - 1 <= 148 // S
+        covered += begins[-1]
+        pos = end
+    assert pos == len(table) and covered == units_total
 
 
 @pytest.mark.parametrize("name", sorted(SHAPE_SETS))
