@@ -162,6 +162,13 @@ flora_status flora_set_decompress_apply(flora_set* set, const uint64_t* seeds, f
 flora_status flora_set_resample_transfer(flora_set* set, const uint64_t* seeds_old, const uint64_t* seeds_new, void* stream);
 /* flora_momentum_step_resampled for every matrix of the set (created with gradients). */
 flora_status flora_set_momentum_step_resampled(flora_set* set, float beta, const uint64_t* seeds_old, const uint64_t* seeds_new, void* stream);
+/* flora_transfer_axpby for every matrix of a set:  dst.S[i] <- b dst.S[i] + a src.S[i] A(seeds_old[i]) A(seeds_new[i])^T.
+ * Feeds the accumulated sketches of Algorithm 1 (the set `src`, projections seeds_old) into the momentum of
+ * Algorithm 2 (the set `dst`, projections seeds_new) with a = (1-beta)/tau, b = beta, in two launches for the
+ * whole model.  Both sets hold the same number of matrices with equal row counts and the same rank
+ * (FLORA_ERR_SHAPE otherwise); m_i and the operand dtype are taken from dst's G (or W).  src may be dst. */
+flora_status flora_set_transfer_axpby(flora_set* dst, const flora_set* src, const uint64_t* seeds_old, const uint64_t* seeds_new,
+                                      float a, float b, void* stream);
 /* Sets every sketch of the set to zero (start of an accumulation cycle, Algorithm 1). */
 flora_status flora_set_zero_state(flora_set* set, void* stream);
 
@@ -179,6 +186,10 @@ int flora_resamples_at(int64_t t, int64_t kappa);
  * End-to-end step with HOST gradients (what a data loader / offloaded backward pass would hand
  * over): copies G (host, ideally pinned) to the set's device gradient buffers, then compresses.
  * ------------------------------------------------------------------------------------------- */
+/* Enqueues on `stream` the host->device copies of host_G[i] (n_i x m_i elements of the set's gradient dtype, densely
+ * packed, ideally pinned) into the set's device gradient buffers; the next compression or momentum step of the
+ * set on that stream then consumes them. */
+flora_status flora_set_upload_gradients(flora_set* set, const void* const* host_G, void* stream);
 /* host_G[i]: host pointer to n_i x m_i elements of the set's gradient dtype, densely packed
  * (ld = m_i).  Enqueues the host->device copies and the compression on `stream`.            */
 flora_status flora_set_compress_accumulate_from_host(flora_set* set, const void* const* host_G,

@@ -27,8 +27,8 @@ EXPORTS = [
     "flora_compress_accumulate", "flora_decompress_apply", "flora_momentum_step", "flora_momentum_step_resampled", "flora_resample_transfer",
     "flora_resample_transfer_static", "flora_transfer_axpby", "flora_materialize_A", "flora_set_create", "flora_set_destroy",
     "flora_set_rebind_gradients", "flora_set_compress_accumulate", "flora_set_momentum_step",
-    "flora_set_decompress_apply", "flora_set_resample_transfer", "flora_set_momentum_step_resampled", "flora_set_zero_state", "flora_derive_seed",
-    "flora_resamples_at", "flora_set_compress_accumulate_from_host", "flora_set_read_weights_to_host",
+    "flora_set_decompress_apply", "flora_set_resample_transfer", "flora_set_transfer_axpby", "flora_set_momentum_step_resampled", "flora_set_zero_state", "flora_derive_seed",
+    "flora_resamples_at", "flora_set_upload_gradients", "flora_set_compress_accumulate_from_host", "flora_set_read_weights_to_host",
     "flora_debug_force_path", "flora_debug_plan", "flora_debug_wait_timeout_selftest", "flora_launch_count", "flora_device_status", "flora_status_string", "flora_version",
 ]
 
@@ -73,11 +73,13 @@ def load() -> ctypes.CDLL:
             "flora_set_decompress_apply": (I32, [P, ctypes.POINTER(U64), F, F, P]),
             "flora_set_resample_transfer": (I32, [P, ctypes.POINTER(U64), ctypes.POINTER(U64), P]),
             "flora_set_momentum_step_resampled": (I32, [P, F, ctypes.POINTER(U64), ctypes.POINTER(U64), P]),
+            "flora_set_transfer_axpby": (I32, [P, P, ctypes.POINTER(U64), ctypes.POINTER(U64), F, F, P]),
             "flora_set_zero_state": (I32, [P, P]),
             "flora_derive_seed": (U64, [U64, U64, U64]),
             "flora_resamples_at": (ctypes.c_int, [I64, I64]),
             "flora_set_compress_accumulate_from_host": (I32, [P, ctypes.POINTER(P), ctypes.POINTER(U64), P]),
             "flora_set_read_weights_to_host": (I32, [P, ctypes.POINTER(P), P]),
+            "flora_set_upload_gradients": (I32, [P, ctypes.POINTER(P), P]),
             "flora_debug_force_path": (None, [ctypes.c_int]),
             "flora_debug_plan": (I32, [P, P, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, P, ctypes.c_int64, P, P]),
             "flora_debug_wait_timeout_selftest": (I32, [P]),
@@ -304,12 +306,21 @@ class FloraSet:
         _check(load().flora_set_resample_transfer(self._h, _u64_array(seeds_old), _u64_array(seeds_new),
                                                   _stream(stream)), "flora_set_resample_transfer")
 
+    def transfer_axpby_from(self, src: "FloraSet", seeds_old: Sequence[int], seeds_new: Sequence[int], a: float, b: float, stream=None) -> None:
+        """self.S[i] <- b self.S[i] + a src.S[i] A(seeds_old[i]) A(seeds_new[i])^T for every matrix."""
+        _check(load().flora_set_transfer_axpby(self._h, src._h, _u64_array(seeds_old), _u64_array(seeds_new), a, b, _stream(stream)),
+               "flora_set_transfer_axpby")
+
     def momentum_step_resampled(self, beta: float, seeds_old: Sequence[int], seeds_new: Sequence[int], stream=None) -> None:
         _check(load().flora_set_momentum_step_resampled(self._h, beta, _u64_array(seeds_old), _u64_array(seeds_new),
                                                         _stream(stream)), "flora_set_momentum_step_resampled")
 
     def zero_state(self, stream=None) -> None:
         _check(load().flora_set_zero_state(self._h, _stream(stream)), "flora_set_zero_state")
+
+    def upload_gradients(self, host_G: Sequence[torch.Tensor], stream=None) -> None:
+        ptrs = (ctypes.c_void_p * self.count)(*[t.data_ptr() for t in host_G])
+        _check(load().flora_set_upload_gradients(self._h, ptrs, _stream(stream)), "flora_set_upload_gradients")
 
     def compress_accumulate_from_host(self, host_G: Sequence[torch.Tensor], seeds: Sequence[int], stream=None) -> None:
         ptrs = (ctypes.c_void_p * self.count)(*[t.data_ptr() for t in host_G])

@@ -398,7 +398,9 @@ flora_status flora_set_decompress_apply(flora_set* set, const uint64_t* seeds, f
     return FLORA_OK;
 }
 
-static flora_status set_transfer(flora_set* set, const uint64_t* seeds_old, const uint64_t* seeds_new, float a, void* stream)
+// dst.S[i] <- b dst.S[i] + a src[i] (A(old_i) A(new_i)^T) for every matrix of the set `dst`.
+static flora_status set_transfer(flora_set* set, const std::vector<flora_mat>& src, const uint64_t* seeds_old, const uint64_t* seeds_new, float a,
+                                 float b, void* stream)
 {
     if (!set || !seeds_old || !seeds_new) return FLORA_ERR_NULL;
     const std::vector<flora_mat>& big = set->has_G ? set->G : set->W;
@@ -412,10 +414,10 @@ static flora_status set_transfer(flora_set* set, const uint64_t* seeds_old, cons
         std::vector<GramJob> jobs;
         for (size_t i = 0; i < set->S.size(); ++i) {
             if (set->S[i].rows == 0) continue;
-            jobs.push_back(GramJob{nullptr, (float*)set->S[i].data, (const float*)set->S[i].data, set->S[i].ld, set->S[i].ld,
+            jobs.push_back(GramJob{nullptr, (float*)set->S[i].data, (const float*)src[i].data, set->S[i].ld, src[i].ld,
                                    (int32_t)set->S[i].rows, (int32_t)big[i].cols, seeds_old[i], seeds_new[i]});
         }
-        return transfer_tc(jobs, r, a, 0.0f, as_stream(stream), g_launches);
+        return transfer_tc(jobs, r, a, b, as_stream(stream), g_launches);
     }
     if (scratch_alloc((void**)&T, sizeof(float) * r * r, as_stream(stream)) != cudaSuccess) {
         cudaGetLastError();
@@ -424,8 +426,7 @@ static flora_status set_transfer(flora_set* set, const uint64_t* seeds_old, cons
     flora_status st = FLORA_OK;
     for (size_t i = 0; i < set->S.size() && st == FLORA_OK; ++i) {
         if (set->S[i].rows == 0) continue;
-        st = transfer_with_scratch(&set->S[i], &set->S[i], big[i].cols, big[i].dtype, seeds_old[i], seeds_new[i], a,
-                                   0.0f, T, as_stream(stream));
+        st = transfer_with_scratch(&set->S[i], &src[i], big[i].cols, big[i].dtype, seeds_old[i], seeds_new[i], a, b, T, as_stream(stream));
     }
     if (cudaFreeAsync(T, as_stream(stream)) != cudaSuccess && st == FLORA_OK) st = FLORA_ERR_CUDA;
     return st;
@@ -433,14 +434,25 @@ static flora_status set_transfer(flora_set* set, const uint64_t* seeds_old, cons
 
 flora_status flora_set_resample_transfer(flora_set* set, const uint64_t* seeds_old, const uint64_t* seeds_new, void* stream)
 {
-    return set_transfer(set, seeds_old, seeds_new, 1.0f, stream);
+    if (!set) return FLORA_ERR_NULL;
+    return set_transfer(set, set->S, seeds_old, seeds_new, 1.0f, 0.0f, stream);
+}
+
+flora_status flora_set_transfer_axpby(flora_set* dst, const flora_set* src, const uint64_t* seeds_old, const uint64_t* seeds_new, float a, float b,
+                                      void* stream)
+{
+    if (!dst || !src) return FLORA_ERR_NULL;
+    if (src->S.size() != dst->S.size() || src->r != dst->r) return FLORA_ERR_SHAPE;
+    for (size_t i = 0; i < dst->S.size(); ++i)
+        if (src->S[i].rows != dst->S[i].rows) return FLORA_ERR_SHAPE;
+    return set_transfer(dst, src->S, seeds_old, seeds_new, a, b, stream);
 }
 
 flora_status flora_set_momentum_step_resampled(flora_set* set, float beta, const uint64_t* seeds_old, const uint64_t* seeds_new, void* stream)
 {
     if (!set || !seeds_old || !seeds_new) return FLORA_ERR_NULL;
     if (!set->has_G) return FLORA_ERR_UNSUPPORTED;
-    flora_status st = set_transfer(set, seeds_old, seeds_new, beta, stream);
+    flora_status st = set_transfer(set, set->S, seeds_old, seeds_new, beta, 0.0f, stream);
     if (st) return st;
     return set_compress(set, seeds_new, 1.0f - beta, 1.0f, stream);
 }
@@ -457,19 +469,30 @@ flora_status flora_set_zero_state(flora_set* set, void* stream)
     return FLORA_OK;
 }
 
-flora_status flora_set_compress_accumulate_from_host(flora_set* set, const void* const* host_G, const uint64_t* seeds, void* stream)
+flora_status flora_set_upload_gradients(flora_set* set, const void* const* host_G, void* stream)
 {
-    if (!set || !host_G || !seeds) return FLORA_ERR_NULL;
+    if (!set || !host_G) return FLORA_ERR_NULL;
     if (!set->has_G) return FLORA_ERR_UNSUPPORTED;
     for (size_t i = 0; i < set->G.size(); ++i) {
         const flora_mat& g = set->G[i];
         if (g.rows == 0 || g.cols == 0) continue;
         if (!host_G[i]) return FLORA_ERR_NULL;
         const size_t es = elem_size(g.dtype);
-        cudaError_t e = cudaMemcpy2DAsync(g.data, es * g.ld, host_G[i], es * g.cols, es * g.cols, (size_t)g.rows,
-                                          cudaMemcpyHostToDevice, as_stream(stream));
+        // a densely stored matrix is one plain copy; a strided one goes row by row
+        cudaError_t e = g.ld == g.cols
+                            ? cudaMemcpyAsync(g.data, host_G[i], es * (size_t)g.rows * (size_t)g.cols, cudaMemcpyHostToDevice, as_stream(stream))
+                            : cudaMemcpy2DAsync(g.data, es * g.ld, host_G[i], es * g.cols, es * g.cols, (size_t)g.rows, cudaMemcpyHostToDevice,
+                                                as_stream(stream));
         if (e != cudaSuccess) return FLORA_ERR_CUDA;
     }
+    return FLORA_OK;
+}
+
+flora_status flora_set_compress_accumulate_from_host(flora_set* set, const void* const* host_G, const uint64_t* seeds, void* stream)
+{
+    if (!seeds) return FLORA_ERR_NULL;
+    flora_status st = flora_set_upload_gradients(set, host_G, stream);
+    if (st) return st;
     return flora_set_compress_accumulate(set, seeds, stream);
 }
 
@@ -482,8 +505,10 @@ flora_status flora_set_read_weights_to_host(flora_set* set, void* const* host_W,
         if (w.rows == 0 || w.cols == 0) continue;
         if (!host_W[i]) return FLORA_ERR_NULL;
         const size_t es = elem_size(w.dtype);
-        cudaError_t e = cudaMemcpy2DAsync(host_W[i], es * w.cols, w.data, es * w.ld, es * w.cols, (size_t)w.rows,
-                                          cudaMemcpyDeviceToHost, as_stream(stream));
+        cudaError_t e = w.ld == w.cols
+                            ? cudaMemcpyAsync(host_W[i], w.data, es * (size_t)w.rows * (size_t)w.cols, cudaMemcpyDeviceToHost, as_stream(stream))
+                            : cudaMemcpy2DAsync(host_W[i], es * w.cols, w.data, es * w.ld, es * w.cols, (size_t)w.rows, cudaMemcpyDeviceToHost,
+                                                as_stream(stream));
         if (e != cudaSuccess) return FLORA_ERR_CUDA;
     }
     return FLORA_OK;

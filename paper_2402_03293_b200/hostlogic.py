@@ -74,3 +74,53 @@ class MomentumState:
             self.ops.momentum_step(self.beta, cur, stream)
         self.ops.decompress_apply(cur, lr, 1.0, stream)
         self.t += 1
+
+
+class AccumulatedMomentum:
+    """Algorithm 1 feeding Algorithm 2: tau micro-steps are compressed into C with the accumulation
+    projections; at the end of the cycle the mean gradient G~ = C A_acc / tau is Algorithm 2's gradient, so
+    M <- beta M + (1-beta)/tau C (A_acc A_mom^T) without ever forming G~, the update M A_mom is applied, C is
+    zeroed and the accumulation projections are resampled (Section 2.4).  Every kappa optimizer steps the
+    momentum projections are resampled too and M is carried over first (Algorithm 2's resampling branch).
+
+    `acc` holds the gradients and C, `mom` holds the weights and M (objects with the methods of
+    :class:`paper_2402_03293_b200.binding.FloraSet`)."""
+
+    def __init__(self, acc, mom, count: int, tau: int, beta: float, kappa: int, base_seed: int = 0):
+        if tau < 1:
+            raise ValueError("tau must be positive")
+        self.acc, self.mom, self.count, self.tau, self.beta, self.kappa = acc, mom, count, tau, beta, kappa
+        self.base_seed = base_seed
+        self.t = 0                      # optimizer steps done
+        self.micro_step = 0
+        self.acc_epoch = 0
+        self.mom_epoch = 0
+
+    def acc_seeds(self) -> List[int]:
+        return [binding.flora_derive_seed(self.base_seed, i, self.acc_epoch) for i in range(self.count)]
+
+    def mom_seeds(self, epoch: int) -> List[int]:
+        return [binding.flora_derive_seed(self.base_seed ^ 0x5DEECE66D, i, epoch) for i in range(self.count)]
+
+    def accumulate(self, stream=None) -> bool:
+        """Compress the gradients currently bound to `acc`; True when the cycle is full."""
+        if self.micro_step >= self.tau:
+            raise RuntimeError("cycle is full: call apply() first")
+        self.acc.compress_accumulate(self.acc_seeds(), stream)
+        self.micro_step += 1
+        return self.micro_step == self.tau
+
+    def apply(self, lr: float, stream=None) -> None:
+        if self.micro_step != self.tau:
+            raise RuntimeError("cycle is not full")
+        if binding.flora_resamples_at(self.t, self.kappa):
+            if self.t > 0:              # M = 0 at t = 0: nothing to carry over
+                self.mom.resample_transfer(self.mom_seeds(self.mom_epoch), self.mom_seeds(self.mom_epoch + 1), stream)
+            self.mom_epoch += 1
+        cur = self.mom_seeds(self.mom_epoch)
+        self.mom.transfer_axpby_from(self.acc, self.acc_seeds(), cur, (1.0 - self.beta) / self.tau, self.beta, stream)
+        self.mom.decompress_apply(cur, lr, 1.0, stream)
+        self.acc.zero_state(stream)
+        self.acc_epoch += 1
+        self.micro_step = 0
+        self.t += 1

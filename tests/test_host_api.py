@@ -139,3 +139,28 @@ def test_momentum_order_algorithm_2():
     assert [c[0] for c in ops3.calls] == ["momentum_step", "decompress_apply"] * 3 + ["momentum_step_resampled", "decompress_apply"]
     fused = ops3.calls[6]
     assert fused[1] == 0.9 and fused[2] == ops3.calls[4][2] and fused[3] == ops3.calls[7][1]
+
+
+def test_accumulation_feeding_momentum_order():
+    acc, mom = _Recorder(), _Recorder()
+    both = hostlogic.AccumulatedMomentum(acc, mom, count=2, tau=3, beta=0.75, kappa=2, base_seed=9)
+    for step in range(3):
+        s_acc = both.acc_seeds()
+        for k in range(3):
+            assert both.accumulate() == (k == 2)
+        with pytest.raises(RuntimeError):
+            both.accumulate()
+        both.apply(0.5)
+        assert both.acc_seeds() != s_acc                           # a fresh accumulation projection per cycle
+    assert [c[0] for c in acc.calls] == (["compress_accumulate"] * 3 + ["zero_state"]) * 3
+    names = [c[0] for c in mom.calls]
+    # t = 0 resamples (nothing to carry), t = 1 keeps the projection, t = 2 resamples and carries M over first
+    assert names == ["transfer_axpby_from", "decompress_apply"] * 2 + ["resample_transfer", "transfer_axpby_from", "decompress_apply"]
+    ax0, ax1, tr, ax2 = mom.calls[0], mom.calls[2], mom.calls[4], mom.calls[5]
+    assert ax0[1] is acc and ax0[2] == acc.calls[0][1]             # the sketches of `acc` with the cycle's accumulation seeds
+    assert ax0[4:6] == (0.25 / 3, 0.75)                            # (1 - beta) / tau and beta
+    assert ax0[3] == ax1[3] == mom.calls[1][1] == tr[1]            # one momentum projection until it is resampled
+    assert tr[2] == ax2[3] == mom.calls[6][1] and tr[2] != tr[1]
+    assert mom.calls[1][2:] == (0.5, 1.0)
+    with pytest.raises(RuntimeError):
+        both.apply(0.5)
