@@ -1,15 +1,17 @@
 #!/usr/bin/env python
 """Benchmark of the Flora hot path on B200: gradient GB/s per Flora step.
 
-A step is one accumulation cycle of Algorithm 1 over the GPT-2-small-shaped weight set
-(12 x {768x2304, 768x768, 768x3072, 3072x768}, bf16, r = 32): tau = 8 compressions
-(C += G A^T, one fresh gradient set each), one decompress-apply (W -= lr/tau * C A) and the
-reset of C.  `value` = gradient bytes consumed per step / device time of the step.
+The default workload is the GPT-2-XL-shaped weight set (48 x {1600x4800, 1600x1600, 1600x6400, 6400x1600}, bf16
+gradients with 1 % outliers, r = 256, tau = 16, beta = 0.9): a step is one accumulation cycle of Algorithm 1 feeding
+Algorithm 2 -- tau compressions C += G A_acc^T (a fresh gradient set each), M <- beta M + (1-beta)/tau C A_acc A_mom^T,
+the update W -= lr M A_mom, and the reset of C.  `value` = gradient bytes consumed per step / device time of the step.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl flora|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl flora|reference] [--workload NAME] [--rank R]
 
-With N > 1 (launched by torch.distributed.run) every rank runs an independent replica of the
-same work on its own GPU (the path has no exchange step); times are the max over ranks.
+Other workloads: an accumulation workload runs tau compressions + one decompress-apply per step; a momentum
+workload runs one momentum step + one decompress-apply per step, with the momentum transfer at the steps
+Algorithm 2 resamples at.  With N > 1 (launched by torch.distributed.run) every rank runs an independent replica of
+the same work on its own GPU (the path has no exchange step); times are the max over ranks.
 """
 from __future__ import annotations
 
@@ -27,36 +29,61 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+from paper_2402_03293_b200 import hostlogic  # noqa: E402
 from paper_2402_03293_b200 import replicas  # noqa: E402
 from paper_2402_03293_b200 import workloads as wl  # noqa: E402
 
-WORKLOAD = "gpt2_small_set"
+DEFAULT_WORKLOAD = "gpt2_xl_set"
 METRIC = "gradient GB/s per Flora step (compress+decompress-apply)"
 LR = 1e-3
-FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
-# (None once a kernel has changed since its counters were taken)
-NCU_TRAFFIC_COMPRESS = 182438144
-NCU_TRAFFIC_DECOMPRESS = 291994368
+FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1400.0
+NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
+MIN_TIMED_SECONDS = 1.5        # the K-step block is repeated until this much device time has been measured
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised
+# under profiles/ (absent = not captured since the kernel last changed)
+NCU_TRAFFIC = {}
 
 
 # ------------------------------------------------------------------------------------------ helpers
-def algorithmic_bytes(w: wl.Workload):
-    """Bytes each operation must move (A costs none: it is regenerated)."""
+def op_costs(w: wl.Workload, r: int):
+    """Algorithmic bytes and flops of each operation over the weight set (A costs no bytes: it is regenerated)."""
     eb = w.elem_bytes
-    state = sum(n * w.r * 4 for n, _ in w.shapes)
-    compress = w.elements * eb + 2 * state            # read G once, read + write C
-    decompress = 2 * w.elements * eb + state          # read + write W, read C
-    return compress, decompress
+    state = sum(n * r * 4 for n, _ in w.shapes)
+    flops = 2 * w.elements * r
+    transfer_flops = sum(2 * r * r * m + 2 * n * r * r for n, m in w.shapes)
+    return {
+        "compress": (w.elements * eb + 2 * state, flops),                 # read G once, read + write the sketch
+        "momentum": (w.elements * eb + 2 * state, flops),
+        "decompress": (2 * w.elements * eb + state, flops),               # read + write W, read the sketch
+        "transfer": (2 * state, transfer_flops),                          # read + write M
+        "transfer_axpby": (3 * state, transfer_flops),                    # read C, read + write M
+        "momentum_resampled": (w.elements * eb + 4 * state, flops + transfer_flops),
+        "zero": (state, 0),
+    }
 
 
-def measured_peak():
+def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+            d = json.load(f)
+        return float(d["hbm_gbs"]), float(d["bf16_tflops_sustained"]), "measured (MEASURED_PEAKS.json: hbm_gbs, bf16_tflops_sustained)"
     except Exception:
-        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s)"
+        return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback (6.65 TB/s, 1.4 PFLOP/s sustained)"
+
+
+def roofline_block(kernel: str, nbytes: int, flops: int, us: float, hbm: float, tf: float, source: str):
+    """Roofline of one launch: the slower of its bytes at the HBM peak and its flops at the tensor peak."""
+    t_hbm, t_tensor = nbytes / (hbm * 1e9) * 1e6, flops / (tf * 1e12) * 1e6
+    nominal_us = max(nbytes / (NOMINAL_HBM_GBS * 1e9), flops / (NOMINAL_BF16_TFLOPS * 1e12)) * 1e6
+    if t_hbm >= t_tensor:
+        bound, achieved, peak, unit = "hbm", nbytes / us / 1e3, hbm, "GB/s"
+    else:
+        bound, achieved, peak, unit = "tensor", flops / us / 1e6, tf, "TFLOP/s"
+    return {"bound": bound, "kernel": kernel, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+            "frac_of_nominal": nominal_us / us, "nominal": "8 TB/s HBM, 2.25 PFLOP/s dense bf16",
+            "bytes_per_launch": nbytes, "flops_per_launch": flops, "us_per_launch": us, "hbm_side_us": t_hbm, "tensor_side_us": t_tensor,
+            "peak_source": source}
 
 
 class ClockSampler:
@@ -91,44 +118,186 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows:
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
+                power.append(float(r[2]))
                 for name, flag in zip(names, r[3:7]):
                     if flag.lower().startswith("active"):
                         reasons.add(name)
             except Exception:
                 continue
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "sm_mhz_min": min(sm) if sm else None, "power_w_max": max(power) if power else None,
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-# ------------------------------------------------------------------------------------------ reference arm
-def oracle_sample_step(w: wl.Workload, layers: int, state):
-    """One Flora step of the CPU oracle over the first `layers` transformer blocks (4 matrices each)."""
-    from oracle import flora_oracle as orc
-    import numpy as np
-    count = 4 * layers
-    if not state:
-        state["G"] = [[wl.as_numpy(wl.gradient(w, i, k)) for i in range(count)] for k in range(w.tau)]
-        state["W"] = [wl.as_numpy(wl.weight(w, i, std=0.02)) for i in range(count)]
-        state["C"] = [np.zeros((w.shapes[i][0], w.r), dtype=np.float32) for i in range(count)]
-        state["epoch"] = 0
-    t0 = time.perf_counter()
-    for i in range(count):
-        n, m = w.shapes[i]
-        A = orc.projection(1000 * state["epoch"] + i, w.r, m, w.dtype)
-        state["C"][i][:] = 0
-        for k in range(w.tau):
-            orc.compress_accumulate(state["G"][k][i], A, state["C"][i])
-        orc.decompress_apply(state["W"][i], state["C"][i], A, LR, 1.0 / w.tau)
-    state["epoch"] += 1
-    dt = time.perf_counter() - t0
-    grad_bytes = w.tau * sum(n * m for n, m in w.shapes[:count]) * w.elem_bytes
-    return dt, grad_bytes
+# ------------------------------------------------------------------------------------------ the step
+class Rotating:
+    """The set operations over a ring of gradient sets that share weights and sketches: every compression takes
+    the next gradient set, so no launch finds its input in L2.  Marks the stream with an event whenever the kind
+    of operation changes (the per-kernel durations of the roofline block come from these marks)."""
+
+    def __init__(self, sets, host_sets=None):
+        self.sets, self.host_sets, self.k = sets, host_sets, 0
+        self._h = sets[0]._h
+        self.marks = None           # list of (kind, event) while a timed block records
+        self.counts = {}
+        self.last = None
+
+    def mark(self, kind):
+        if self.marks is not None:
+            self.counts[kind] = self.counts.get(kind, 0) + 1
+            if kind != self.last:
+                ev = torch.cuda.Event(enable_timing=True)
+                ev.record()
+                self.marks.append((kind, ev))
+                self.last = kind
+
+    def _next(self):
+        s = self.sets[self.k % len(self.sets)]
+        if self.host_sets is not None:          # end-to-end leg: this micro-step's gradients come from pinned host memory
+            s.upload_gradients(self.host_sets[self.k % len(self.host_sets)])
+        self.k += 1
+        return s
+
+    def compress_accumulate(self, seeds, stream=None):
+        self.mark("compress")
+        self._next().compress_accumulate(seeds, stream)
+
+    def momentum_step(self, beta, seeds, stream=None):
+        self.mark("momentum")
+        self._next().momentum_step(beta, seeds, stream)
+
+    def momentum_step_resampled(self, beta, old, new, stream=None):
+        self.mark("momentum_resampled")
+        self._next().momentum_step_resampled(beta, old, new, stream)
+
+    def resample_transfer(self, old, new, stream=None):
+        self.mark("transfer")
+        self.sets[0].resample_transfer(old, new, stream)
+
+    def transfer_axpby_from(self, src, old, new, a, b, stream=None):
+        self.mark("transfer_axpby")
+        self.sets[0].transfer_axpby_from(src, old, new, a, b, stream)
+
+    def decompress_apply(self, seeds, lr, scale, stream=None):
+        self.mark("decompress")
+        self.sets[0].decompress_apply(seeds, lr, scale, stream)
+
+    def zero_state(self, stream=None):
+        self.mark("zero")
+        self.sets[0].zero_state(stream)
+
+
+def make_stepper(w: wl.Workload, acc: Rotating, mom, count: int, base_seed: int):
+    """One Flora step of the workload's mode as a closure, sequenced by the host classes of Algorithms 1 and 2."""
+    if w.mode == "accumulate":
+        cyc = hostlogic.AccumulationCycle(acc, count, w.tau, base_seed)
+
+        def step():
+            for _ in range(w.tau):
+                cyc.accumulate()
+            cyc.apply(LR)
+        return step, f"{w.tau} x compress_accumulate + decompress_apply + zero C"
+    if w.mode == "momentum":
+        st = hostlogic.MomentumState(acc, count, w.beta, w.kappa, base_seed)
+        n = [0]
+
+        def step():
+            # resampling at every step multiplies the state by about sqrt(m/r) each time: restart it every fourth step
+            if w.kappa == 1 and n[0] % 4 == 0:
+                acc.zero_state()
+            st.step(LR)
+            n[0] += 1
+        what = "momentum_step + decompress_apply"
+        what += (", with the transfer fused into every step (kappa = 1; M restarts from zero every 4th step)" if w.kappa == 1
+                 else f"; resampling + transfer every {w.kappa} steps")
+        return step, what
+    both = hostlogic.AccumulatedMomentum(acc, mom, count, w.tau, w.beta, w.kappa, base_seed)
+
+    def step():
+        for _ in range(w.tau):
+            both.accumulate()
+        both.apply(LR)
+    return step, (f"{w.tau} x compress_accumulate into C + transfer_axpby (M <- beta M + (1-beta)/tau C A_acc A_mom^T) + "
+                  f"decompress_apply of M + zero C; M resampled every {w.kappa} steps")
+
+
+# ------------------------------------------------------------------------------------------ reference arm (CPU oracle)
+class OracleSample:
+    """The workload's step on a sample of rows of the first transformer block's matrices, on the CPU oracle."""
+
+    def __init__(self, w: wl.Workload, r: int, rows: int):
+        import numpy as np
+        self.np, self.w, self.r = np, w, r
+        block = 4 if "gpt2" in w.name else (7 if "t5" in w.name else 1)
+        self.ids = list(range(min(block, len(w.shapes))))
+        self.rows = [min(rows, w.shapes[i][0]) for i in self.ids]
+        self.micro = max(1, w.tau)
+        self.G = [[wl.as_numpy(wl.gradient(w, i, k))[:n].copy() for i, n in zip(self.ids, self.rows)] for k in range(min(self.micro, 2))]
+        self.W = [wl.as_numpy(wl.weight(w, i, std=0.02))[:n].copy() for i, n in zip(self.ids, self.rows)]
+        self.C = [np.zeros((n, r), dtype=np.float32) for n in self.rows]
+        self.M = [np.zeros((n, r), dtype=np.float32) for n in self.rows]
+        self.t = 0
+
+    def grad_bytes(self):
+        return self.micro * sum(n * self.w.shapes[i][1] for i, n in zip(self.ids, self.rows)) * self.w.elem_bytes
+
+    def step(self):
+        from oracle import flora_oracle as orc
+        w, r, t = self.w, self.r, self.t
+        t0 = time.perf_counter()
+        for j, i in enumerate(self.ids):
+            m = w.shapes[i][1]
+            if w.mode == "accumulate":
+                A = orc.projection(1000 * t + i, r, m, w.dtype)
+                self.C[j][:] = 0
+                for k in range(w.tau):
+                    orc.compress_accumulate(self.G[k % len(self.G)][j], A, self.C[j])
+                orc.decompress_apply(self.W[j], self.C[j], A, LR, 1.0 / w.tau)
+            elif w.mode == "momentum":
+                epoch = t // w.kappa if w.kappa else 0
+                A = orc.projection(1000 * epoch + i, r, m, w.dtype)
+                if w.kappa and t % w.kappa == 0 and t > 0:
+                    if w.kappa == 1 and t % 4 == 0:
+                        self.M[j][:] = 0
+                    A_old = orc.projection(1000 * (epoch - 1) + i, r, m, w.dtype)
+                    orc.momentum_step_resampled(self.G[0][j], A_old, A, w.beta, self.M[j])
+                else:
+                    orc.momentum_step(self.G[0][j], A, w.beta, self.M[j])
+                orc.decompress_apply(self.W[j], self.M[j], A, LR, 1.0)
+            else:
+                A_acc = orc.projection(1000 * t + i, r, m, w.dtype)
+                A_mom = orc.projection(7_000_000 + i, r, m, w.dtype)
+                self.C[j][:] = 0
+                for k in range(w.tau):
+                    orc.compress_accumulate(self.G[k % len(self.G)][j], A_acc, self.C[j])
+                orc.transfer_axpby(self.M[j], self.C[j], A_acc, A_mom, (1.0 - w.beta) / w.tau, w.beta)
+                orc.decompress_apply(self.W[j], self.M[j], A_mom, LR, 1.0)
+        self.t += 1
+        return time.perf_counter() - t0
+
+    def describe(self):
+        names = ", ".join(f"{n} of {self.w.shapes[i][0]} rows of a {self.w.shapes[i][0]}x{self.w.shapes[i][1]} matrix" for i, n in zip(self.ids, self.rows))
+        return f"the whole step on the first rows of one transformer block's matrices ({names}); GB/s is per row processed, so it extrapolates linearly"
+
+
+def sized_oracle_sample(w: wl.Workload, r: int, seconds_per_step: float) -> OracleSample:
+    """A sample whose step takes about `seconds_per_step` on this host (sized from a small probe)."""
+    probe = OracleSample(w, r, 16)
+    dt = probe.step()
+    rows = int(max(8, min(max(n for n, _ in w.shapes), 16 * seconds_per_step / max(dt, 1e-4))))
+    return OracleSample(w, r, rows)
+
+
+def select_workload(args):
+    w = wl.WORKLOADS[args.workload]
+    r = args.rank or w.r
+    return w, r
 
 
 def run_reference(args):
@@ -136,24 +305,20 @@ def run_reference(args):
     if rank != 0:
         return
     from oracle import flora_oracle as orc
-    w = wl.WORKLOADS[WORKLOAD]
-    layers = 4
-    state = {}
+    w, r = select_workload(args)
+    # the whole run (warm-up + steps) should end within about two minutes
+    per_step = max(0.05, min(3.0, 120.0 / max(1, args.steps + args.warmup)))
+    sample = sized_oracle_sample(w, r, per_step)
     for _ in range(args.warmup):
-        oracle_sample_step(w, layers, state)
-    total_t, total_b = 0.0, 0
-    for _ in range(args.steps):
-        dt, b = oracle_sample_step(w, layers, state)
-        total_t += dt
-        total_b += b
-    value = total_b / total_t / 1e9
-    sample = f"each step: one full cycle (tau={w.tau} compress + 1 decompress-apply) over {layers} of 12 transformer blocks (4 matrices)"
+        sample.step()
+    total_t = sum(sample.step() for _ in range(args.steps))
+    value = sample.grad_bytes() * args.steps / total_t / 1e9
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "r": w.r, "tau": w.tau, "matrices": 4 * layers, "note": "CPU oracle on host cores, bounded sample"},
-        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": orc.max_threads(), "kind": "oracle", "sample": sample},
+        "config": {"workload": w.name, "r": r, "tau": w.tau, "mode": w.mode, "note": "CPU oracle on host cores, bounded sample per step"},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": orc.max_threads(), "kind": "oracle", "sample": sample.describe()},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
@@ -182,31 +347,44 @@ def run_flora(args):
         torch.cuda.synchronize()
 
     fb.load()
-    w = wl.WORKLOADS[WORKLOAD]
+    w, r = select_workload(args)
+    if w.dtype != "bf16":
+        raise RuntimeError("the benchmark runs the bf16 workloads; the fp32 single matrix is a parity case")
     count = len(w.shapes)
-    # tau gradient sets (1.36 GB in total, far larger than the 126 MB L2), weights, sketches
-    G = [[wl.gradient(w, i, k, device=dev, base_seed=rank) for i in range(count)] for k in range(w.tau)]
+    grad_set_bytes = w.elements * w.elem_bytes
+    # gradient sets that rotate: together far larger than the 126 MB L2 (at least 1 GB), at most tau of them
+    n_sets = max(2, min(max(w.tau, 4), -(-(1 << 30) // grad_set_bytes)))
+    if grad_set_bytes > (2 << 30):
+        n_sets = 4
+    G = [[wl.gradient(w, i, k, device=dev, base_seed=rank) for i in range(count)] for k in range(n_sets)]
     W = [wl.weight(w, i, device=dev, std=0.02) for i in range(count)]
-    C = [torch.zeros(n, w.r, device=dev) for n, _ in w.shapes]
-    sets = [fb.FloraSet(G[k], W, C) for k in range(w.tau)]
-    epoch = [0]
+    C = [torch.zeros(n, r, device=dev) for n, _ in w.shapes]
+    both = w.mode == "accumulate+momentum"
+    M = [torch.zeros(n, r, device=dev) for n, _ in w.shapes] if both else None
+    sets = [fb.FloraSet(G[k], None if both else W, C) for k in range(n_sets)]
+    mset = fb.FloraSet(None, W, M) if both else None
+    acc = Rotating(sets)
+    mom = Rotating([mset]) if both else None
+    step, what = make_stepper(w, acc, mom, count, base_seed=17 + rank)
 
-    def seeds():
-        return fb.seed_array([fb.flora_derive_seed(17, i, epoch[0]) for i in range(count)])
+    def begin_marks():
+        for rot in (acc, mom):
+            if rot is not None:
+                rot.marks, rot.counts, rot.last = shared_marks, shared_counts, None
 
-    def step(marks=None):
-        s = seeds()
-        if marks is not None:
-            marks[0].record()
-        for k in range(w.tau):
-            sets[k].compress_accumulate(s)
-        if marks is not None:
-            marks[1].record()
-        sets[0].decompress_apply(s, LR, 1.0 / w.tau)
-        if marks is not None:
-            marks[2].record()
-        sets[0].zero_state()
-        epoch[0] += 1
+    def timed_block(k):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(k):
+            step()
+            end = torch.cuda.Event(enable_timing=True)
+            end.record()
+            shared_marks.append(("end", end))
+            for rot in (acc, mom):
+                if rot is not None:
+                    rot.last = None
+        e1.record()
+        return e0, e1
 
     for _ in range(args.warmup):
         step()
@@ -215,99 +393,121 @@ def run_flora(args):
     if rank == 0:
         sampler.start()
     launches0 = fb.flora_launch_count()
-    # three event marks per step inside the timed region: before the compressions, between them and the
-    # decompression, after it (per-kernel durations for the roofline block come from these)
-    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(args.steps):
-        step(marks[i])
-    e1.record()
-    barrier()
-    launches = fb.flora_launch_count() - launches0
+    shared_marks, shared_counts = [], {}
+    begin_marks()
+    # K steps form a block; blocks repeat until enough device time has been measured; the median block is reported
+    blocks, spent = [], 0.0
+    while True:
+        e0, e1 = timed_block(args.steps)
+        barrier()
+        blocks.append(e0.elapsed_time(e1))
+        spent += blocks[-1] * 1e-3
+        done = spent >= MIN_TIMED_SECONDS or len(blocks) >= 200
+        if dist:                        # all ranks stop together
+            flag = torch.tensor([1.0 if done else 0.0], device=dev)
+            dist.all_reduce(flag, op=dist.ReduceOp.MAX)
+            done = bool(flag.item())
+        if done:
+            break
+    launches_per_block = (fb.flora_launch_count() - launches0) // len(blocks)
     clocks = sampler.stop() if rank == 0 else None
+    for rot in (acc, mom):
+        if rot is not None:
+            rot.marks = None
     if fb.flora_device_status() != 0:
         raise RuntimeError("a device-side wait timed out during the timed region")
-    grad_bytes_step = w.tau * w.elements * w.elem_bytes
-    agg = replicas.aggregate_throughput(grad_bytes_step, args.steps, e0.elapsed_time(e1), dist, dev)
+    grad_bytes_step = (w.tau if w.mode != "momentum" else 1) * grad_set_bytes
+    agg = replicas.aggregate_throughput(grad_bytes_step, args.steps, statistics.median(blocks), dist, dev)
     ms, value = agg["ms"], agg["gbs"]
 
-    comp_bytes, dec_bytes = algorithmic_bytes(w)
-    c_avg = sum(m[0].elapsed_time(m[1]) for m in marks) / (args.steps * w.tau)     # ms per compress launch
-    d_avg = sum(m[1].elapsed_time(m[2]) for m in marks) / args.steps              # ms per decompress launch
-    peak, peak_src = measured_peak()
-    comp_gbs, dec_gbs = comp_bytes / (c_avg * 1e-3) / 1e9, dec_bytes / (d_avg * 1e-3) / 1e9
-    step_roof_ms = (w.tau * comp_bytes + dec_bytes) / (peak * 1e9) * 1e3
-    roofline = {"bound": "hbm", "kernel": "compress_tc_kernel (C += G A^T), one launch over the weight set, 8 launches per step",
-                "achieved": comp_gbs, "peak": peak, "unit": "GB/s", "frac": comp_gbs / peak, "traffic": NCU_TRAFFIC_COMPRESS,
-                "peak_source": peak_src, "bytes_per_launch": comp_bytes, "us_per_launch": 1e3 * c_avg,
-                "decompress_apply": {"kernel": "decompress_tc_kernel", "achieved": dec_gbs, "frac": dec_gbs / peak,
-                                     "bytes_per_launch": dec_bytes, "us_per_launch": 1e3 * d_avg, "traffic": NCU_TRAFFIC_DECOMPRESS},
-                "step_frac_of_roofline": step_roof_ms / (ms / args.steps)}
+    # per-operation durations from the marks recorded inside the timed blocks
+    spent_ms, kinds = {}, {}
+    for (k0, ev0), (_, ev1) in zip(shared_marks, shared_marks[1:]):
+        if k0 != "end":
+            spent_ms[k0] = spent_ms.get(k0, 0.0) + ev0.elapsed_time(ev1)
+    for k, total in spent_ms.items():
+        kinds[k] = 1e3 * total / shared_counts[k]                    # microseconds per launch group of that kind
+    costs = op_costs(w, r)
+    hbm, tf, src = measured_peaks()
+    names = {"compress": "compress kernel (C += G A^T), one launch over the weight set", "momentum": "compress kernel as the momentum update",
+             "momentum_resampled": "gram + apply + compress kernels (Algorithm 2's resampling step)",
+             "decompress": "decompress_tc_kernel (W -= lr S A), one launch over the weight set",
+             "transfer": "gram + apply kernels (M <- M A_old A_new^T)", "transfer_axpby": "gram + apply kernels (M <- beta M + a C A_acc A_mom^T)"}
+    main_kind = "compress" if "compress" in kinds else ("momentum" if "momentum" in kinds else "momentum_resampled")
+    roofline = roofline_block(names[main_kind], costs[main_kind][0], costs[main_kind][1], kinds[main_kind], hbm, tf, src)
+    roofline["launches_per_step"] = shared_counts[main_kind] // (args.steps * len(blocks))
+    roofline["traffic"] = NCU_TRAFFIC.get((w.name, r, main_kind))
+    roofline["other_kernels"] = {k: roofline_block(names[k], costs[k][0], costs[k][1], us, hbm, tf, src) | {"traffic": NCU_TRAFFIC.get((w.name, r, k))}
+                                 for k, us in kinds.items() if k in names and k != main_kind}
+    step_bound_us = sum(max(costs[k][0] / (hbm * 1e9), costs[k][1] / (tf * 1e12)) * 1e6 * shared_counts[k] for k in kinds if k in costs) \
+        / (args.steps * len(blocks))
+    roofline["step_frac_of_roofline"] = step_bound_us / (1e3 * ms / args.steps)
 
-    # end to end: gradients start in pinned host memory, the updated weights are read back
-    e2e = None
-    e2e_steps = max(1, min(args.steps, 3))
-    hostG = [[g.cpu().pin_memory() for g in G[k]] for k in range(w.tau)]
+    # end to end: every micro-step's gradients start in pinned host memory, the updated weights are read back
+    e2e_steps = 2 if grad_bytes_step > (8 << 30) else max(1, min(args.steps, 3))
+    n_host = min(n_sets, 2)
+    hostG = [[g.cpu().pin_memory() for g in G[k]] for k in range(n_host)]
     hostW = [torch.empty(n, m, dtype=wl.torch_dtype(w.dtype)).pin_memory() for n, m in w.shapes]
-
+    acc.host_sets = hostG
+    wset = mset if both else sets[0]
     # the read-back of a step's weights runs on a second stream, so it shares the (full-duplex) link with the next
     # step's uploads; it must have finished before the next decompression overwrites the weights
-    main, side = torch.cuda.current_stream(), torch.cuda.Stream()
+    main_stream, side = torch.cuda.current_stream(), torch.cuda.Stream()
     updated, read_back = torch.cuda.Event(), torch.cuda.Event()
     read_back.record(side)
 
     def e2e_step():
-        s = seeds()
-        for k in range(w.tau):
-            sets[k].compress_accumulate_from_host(hostG[k], s)
-        main.wait_event(read_back)
-        sets[0].decompress_apply(s, LR, 1.0 / w.tau)
-        updated.record(main)
+        main_stream.wait_event(read_back)
+        step()
+        updated.record(main_stream)
         side.wait_event(updated)
-        sets[0].read_weights_to_host(hostW, stream=side)
+        wset.read_weights_to_host(hostW, stream=side)
         read_back.record(side)
-        sets[0].zero_state()
-        epoch[0] += 1
 
     e2e_step()
     barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(e2e_steps):
         e2e_step()
-    main.wait_event(read_back)              # the last step's weights have arrived in host memory
+    main_stream.wait_event(read_back)              # the last step's weights have arrived in host memory
     e1.record()
     barrier()
+    acc.host_sets = None
     e2e_agg = replicas.aggregate_throughput(grad_bytes_step, e2e_steps, e0.elapsed_time(e1), dist, dev)
-    e2e = {"value": e2e_agg["gbs"], "unit": "GB/s",
-           "h2d_bytes_per_step": grad_bytes_step, "d2h_bytes_per_step": w.elements * w.elem_bytes, "steps": e2e_steps}
+    e2e = {"value": e2e_agg["gbs"], "unit": "GB/s", "h2d_bytes_per_step": grad_bytes_step,
+           "d2h_bytes_per_step": w.elements * w.elem_bytes, "steps": e2e_steps,
+           "api": "flora_set_upload_gradients + the step's set calls + flora_set_read_weights_to_host, pinned host buffers"}
 
     cpu_baseline = None
     if rank == 0 and world == 1:
         from oracle import flora_oracle as orc
-        state = {}
-        dt, b = oracle_sample_step(w, 12, state)
-        cycles = 1
-        while dt < 10.0 and cycles < 12:                       # about 10 s of oracle work, whole cycles only
-            dt2, b2 = oracle_sample_step(w, 12, state)
-            dt, b, cycles = dt + dt2, b + b2, cycles + 1
-        cpu_baseline = {"value": b / dt / 1e9, "unit": "GB/s", "cores": orc.max_threads(), "kind": "oracle",
-                        "sample": f"{cycles} full cycle(s) (tau={w.tau} compress + decompress-apply) over all 48 matrices, {dt:.1f} s wall"}
+        sample = sized_oracle_sample(w, r, 4.0)
+        total_t, n_steps = 0.0, 0
+        while total_t < 10.0 and n_steps < 6:
+            total_t += sample.step()
+            n_steps += 1
+        cpu_baseline = {"value": sample.grad_bytes() * n_steps / total_t / 1e9, "unit": "GB/s", "cores": orc.max_threads(), "kind": "oracle",
+                        "sample": f"{n_steps} step(s), {total_t:.1f} s wall: " + sample.describe()}
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "matrices": count, "r": w.r, "tau": w.tau, "elements": w.elements,
-                       "step": "8 x compress_accumulate + decompress_apply + zero C",
-                       "l2": "inputs larger than L2: 8 rotating gradient sets, 1.36 GB per step",
+            "config": {"workload": w.name, "matrices": count, "r": r, "tau": w.tau, "beta": w.beta, "kappa": w.kappa, "elements": w.elements,
+                       "step": what,
+                       "l2": f"inputs larger than L2: {n_sets} rotating gradient sets of {grad_set_bytes / 1e9:.2f} GB, a different one per compression",
+                       "timed": f"{len(blocks)} block(s) of {args.steps} steps, {spent:.2f} s of device time; value is the median block",
                        "multi_gpu": "independent replicas, no collective"},
-            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches_per_block), "clocks": clocks,
+            "ms_x_mhz_per_step": (ms / args.steps) * clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None,
         }
         print(json.dumps(line), flush=True)
     for s in sets:
         s.close()
+    if mset:
+        mset.close()
     if dist:
         dist.destroy_process_group()
 
@@ -315,9 +515,11 @@ def run_flora(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="flora", choices=["flora", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=[n for n in wl.CONFIG_ORDER if wl.WORKLOADS[n].dtype == "bf16"])
+    ap.add_argument("--rank", type=int, default=0, help="rank r of the sketches (default: the workload's)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "flora" else args.warmup
     if args.impl == "reference":

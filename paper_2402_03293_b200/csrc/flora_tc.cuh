@@ -54,6 +54,21 @@ struct K2Item {          // one CTA of the decompression kernel
     int32_t tiles;       // 128-row tiles handled
 };
 
+// Position in a ring of `n` stages: stage index and how often the ring has wrapped (its parity is the phase bit of
+// the stage's barriers).  Advanced by one step at a time: the loops that use it run once per 64-column step in a single
+// thread on the critical path, where a division by a run-time value costs more than the MMAs it feeds.
+struct RingPos {
+    int s = 0;
+    uint32_t wraps = 0;
+    __device__ __forceinline__ void advance(int n)
+    {
+        if (++s == n) {
+            s = 0;
+            ++wraps;
+        }
+    }
+};
+
 constexpr int SEEDS_PER_LAUNCH = 448;
 struct SeedTable {
     uint64_t s[SEEDS_PER_LAUNCH];
@@ -148,9 +163,10 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
         if (lane == 0 && item.tiles > 0) {
             ptx::prefetch_tensormap(&mat->map_g);
             int issued = 0;
-            for (int ks = 0; ks < item.ksteps; ++ks) {
-                const int s = ks % gstages, it = ks / gstages;
-                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->empty_g[s]), (it & 1) ^ 1, abort)) break;
+            RingPos pg;
+            for (int ks = 0; ks < item.ksteps; ++ks, pg.advance(gstages)) {
+                const int s = pg.s;
+                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->empty_g[s]), (pg.wraps & 1u) ^ 1u, abort)) break;
                 const uint32_t bar = ptx::smem_addr(&ctl->full_g[s]);
                 ptx::mbar_arrive_expect_tx(bar, (uint32_t)item.tiles * G_TILE_BYTES);
                 for (int t = 0; t < item.tiles; ++t)
@@ -169,10 +185,11 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
             const uint32_t idesc = ptx::umma_idesc_bf16((uint32_t)r_pad);
             const uint64_t desc_base = ptx::umma_desc_k_sw128(smem_base);
             bool ok = true;
-            for (int ks = 0; ks < item.ksteps && ok; ++ks) {
-                const int sg = ks % gstages, sa = ks % astages;
-                const uint32_t pa = (uint32_t)(ks / astages) & 1u;
-                ok = (item.tiles == 0 || ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[sg]), (uint32_t)(ks / gstages) & 1u, abort)) &&
+            RingPos rg, ra;
+            for (int ks = 0; ks < item.ksteps && ok; ++ks, rg.advance(gstages), ra.advance(astages)) {
+                const int sg = rg.s, sa = ra.s;
+                const uint32_t pa = ra.wraps & 1u;
+                ok = (item.tiles == 0 || ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[sg]), rg.wraps & 1u, abort)) &&
                      (S > 1 ? ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->full_a[sa]), pa, abort)
                             : ptx::mbar_wait(ptx::smem_addr(&ctl->full_a[sa]), pa, abort));
                 if (!ok) break;
@@ -200,9 +217,10 @@ compress_tc_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict__
         // ------------------------------------------------------------------ forwarder: this CTA's slice of A to the peers
         if (lane == 0 && S > 1) {
             const uint32_t slice_bytes = (uint32_t)(r_pad / S) * 128u;
-            for (int ks = 0; ks < item.ksteps; ++ks) {
-                const int s = ks % astages, it = ks / astages;
-                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->slice_ready[s]), it & 1, abort)) break;
+            RingPos ra;
+            for (int ks = 0; ks < item.ksteps; ++ks, ra.advance(astages)) {
+                const int s = ra.s;
+                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->slice_ready[s]), ra.wraps & 1u, abort)) break;
                 const uint32_t fbar = ptx::smem_addr(&ctl->full_a[s]);
                 const uint32_t src = a_ring + s * a_bytes + rank * slice_bytes;
                 ptx::mbar_arrive_expect_tx(fbar, (uint32_t)(S - 1) * slice_bytes);   // own slice is in place; peers' bytes to come
@@ -496,14 +514,15 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         // ------------------------------------------------------------------ W tile loads
         if (lane == 0) {
             int gt = 0, pending_from = 0;                       // tiles issued so far over all items of this CTA
+            RingPos pw;
             bool ok = true;
             for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
                 const K2Item item = items[it];
                 const TcMatrix* mat = mats + item.mat;
                 const int live_boxes = min(boxes, (mat->m - item.col0 + 63) >> 6);
-                for (int i = 0; i < item.tiles; ++i, ++gt) {
-                    const int s = gt % slots;
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->w_free[s]), ((gt / slots) & 1) ^ 1, abort);
+                for (int i = 0; i < item.tiles; ++i, ++gt, pw.advance(slots)) {
+                    const int s = pw.s;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->w_free[s]), (pw.wraps & 1u) ^ 1u, abort);
                     if (!ok) break;
                     const uint32_t bar = ptx::smem_addr(&ctl->w_full[s]);
                     ptx::mbar_arrive_expect_tx(bar, (uint32_t)live_boxes * W_BOX_BYTES);
@@ -520,18 +539,21 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         // ------------------------------------------------------------------ S chunk loads (fp32 rows, 32 columns each)
         if (lane == 0) {
             int gc = 0;
+            RingPos pc;
             bool ok = true;
             for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
                 const K2Item item = items[it];
                 const TcMatrix* mat = mats + item.mat;
-                for (int c = 0; c < item.tiles * kchunks; ++c, ++gc) {
-                    const int s = gc % cstages;
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_empty[s]), ((gc / cstages) & 1) ^ 1, abort);
-                    if (!ok) break;
-                    const uint32_t bar = ptx::smem_addr(&ctl->c_full[s]);
-                    ptx::mbar_arrive_expect_tx(bar, S_CHUNK_BYTES);
-                    if (BF16S) ptx::tma_load_2d(c_ring + s * S_CHUNK_BYTES, &mat->map_sb, (c % kchunks) * 64, item.row0 + (c / kchunks) * 128, bar);
-                    else ptx::tma_load_2d(c_ring + s * S_CHUNK_BYTES, &mat->map_s, (c % kchunks) * 32, item.row0 + (c / kchunks) * 128, bar);
+                for (int i = 0; i < item.tiles && ok; ++i) {
+                    for (int kc = 0; kc < kchunks; ++kc, ++gc, pc.advance(cstages)) {
+                        const int s = pc.s;
+                        ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_empty[s]), (pc.wraps & 1u) ^ 1u, abort);
+                        if (!ok) break;
+                        const uint32_t bar = ptx::smem_addr(&ctl->c_full[s]);
+                        ptx::mbar_arrive_expect_tx(bar, S_CHUNK_BYTES);
+                        if (BF16S) ptx::tma_load_2d(c_ring + s * S_CHUNK_BYTES, &mat->map_sb, kc * 64, item.row0 + i * 128, bar);
+                        else ptx::tma_load_2d(c_ring + s * S_CHUNK_BYTES, &mat->map_s, kc * 32, item.row0 + i * 128, bar);
+                    }
                 }
             }
             if (*abort)
@@ -543,10 +565,11 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
             const uint32_t idesc = BF16S ? ptx::umma_idesc_bf16((uint32_t)bn) : ptx::umma_idesc_tf32((uint32_t)bn);
             const uint64_t desc_ring = ptx::umma_desc_k_sw128(c_ring);
             int gt = 0, gc = 0, k = 0;
+            RingPos pc;
             bool ok = true;
             for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++k) {
                 const K2Item item = items[it];
-                const int sb = k % nslabs, sphase = (k / nslabs) & 1;
+                const int sb = nslabs == 2 ? (k & 1) : 0, sphase = (nslabs == 2 ? (k >> 1) : k) & 1;
                 const uint64_t desc_slab = ptx::umma_desc_k_sw128(slab0 + sb * slab_bytes);
                 ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_full[sb]), sphase, abort);
                 // the combine warps' share: of the first slab, or of every slab when there is only one buffer
@@ -554,9 +577,9 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
                 for (int i = 0; i < item.tiles && ok; ++i, ++gt) {
                     const uint32_t acc_addr = tmem + (gt & 1) * bn;
                     ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[gt & 1]), ((gt >> 1) & 1) ^ 1, abort);
-                    for (int kc = 0; kc < kchunks && ok; ++kc, ++gc) {
-                        const int s = gc % cstages;
-                        ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[s]), (gc / cstages) & 1, abort);
+                    for (int kc = 0; kc < kchunks && ok; ++kc, ++gc, pc.advance(cstages)) {
+                        const int s = pc.s;
+                        ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[s]), pc.wraps & 1u, abort);
                         if (!ok) break;
                         ptx::tc_fence_after_sync();
 #pragma unroll
@@ -578,15 +601,17 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         // ------------------------------------------------------------------ W tile stores
         if (lane == 0) {
             int gt = 0;
+            RingPos pw;
+            int prev_slot = 0;
             bool ok = true;
             const bool lag = slots >= 4;               // with few slots, freeing a slot one tile late costs more than it gains
             for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
                 const K2Item item = items[it];
                 const TcMatrix* mat = mats + item.mat;
                 const int live_boxes = min(boxes, (mat->m - item.col0 + 63) >> 6);
-                for (int i = 0; i < item.tiles; ++i, ++gt) {
-                    const int s = gt % slots;
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->out_ready[s]), (gt / slots) & 1, abort);
+                for (int i = 0; i < item.tiles; ++i, ++gt, pw.advance(slots)) {
+                    const int s = pw.s;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->out_ready[s]), pw.wraps & 1u, abort);
                     if (!ok) break;
                     for (int bx = 0; bx < live_boxes; ++bx)
                         ptx::tma_store_2d(&mat->map_w, item.col0 + bx * 64, item.row0 + i * 128, w_ring + s * slot_bytes + bx * W_BOX_BYTES);
@@ -594,7 +619,8 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
                     if (lag) {
                         // one store stays in flight: wait until all but the newest have read their slot, free that one
                         ptx::tma_store_wait_read<1>();
-                        if (gt > 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[(gt - 1) % slots]));
+                        if (gt > 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[prev_slot]));
+                        prev_slot = s;
                     } else {
                         ptx::tma_store_wait_read<0>();          // the slot has been read out: it can be refilled
                         ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[s]));
@@ -602,7 +628,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
                 }
             }
             ptx::tma_store_wait_read<0>();
-            if (lag && gt > 0 && ok) ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[(gt - 1) % slots]));
+            if (lag && gt > 0 && ok) ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[prev_slot]));
             ptx::tma_store_wait_all<0>();
         }
     } else if ((warp >= 2 && warp <= 5) || (warp >= 8 && warp <= 11)) {
@@ -615,6 +641,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         const int row = quarter * 32 + lane;
         const int per_half = boxes << 1;                       // 16-column chunks per half: 2 (bn 64) or 4 (bn 128)
         int gt = 0;
+        RingPos pw;
         bool ok = true;
         const int helper = (half * 4 + (warp - (half ? 8 : 2))) * 32 + lane;              // 0 .. 255
         int k = 0;
@@ -623,7 +650,7 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
             if (k == 0 || nslabs == 1) {
                 // Nothing to combine yet (first item), or a single slab buffer whose refill nothing overlaps: write a
                 // share of the slab alongside the generator warps.
-                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_empty[0]), ((k / nslabs) & 1) ^ 1, abort);
+                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_empty[0]), (((nslabs == 2 ? (k >> 1) : k) & 1) ^ 1), abort);
                 if (!ok) break;
                 k2_generate_slab<BF16S>(slab0, slab_block, kchunks, bn, item.col0, r, make_key(seeds.s[item.mat - seed_base]), scale,
                                         32 * GW + helper, 32 * (GW + K2_HELPER_WARPS));
@@ -634,10 +661,10 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
             const int live_chunks = min(boxes, (mats[item.mat].m - item.col0 + 63) >> 6) << 2;
             const int c_begin = half * per_half;
             const int mine = max(0, min(per_half, live_chunks - c_begin));
-            for (int i = 0; i < item.tiles; ++i, ++gt) {
-                const int s = gt % slots;
+            for (int i = 0; i < item.tiles; ++i, ++gt, pw.advance(slots)) {
+                const int s = pw.s;
                 ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[gt & 1]), (gt >> 1) & 1, abort) &&
-                     ptx::mbar_wait(ptx::smem_addr(&ctl->w_full[s]), (gt / slots) & 1, abort);
+                     ptx::mbar_wait(ptx::smem_addr(&ctl->w_full[s]), pw.wraps & 1u, abort);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t wrow = w_ring + s * slot_bytes + row * 128;
@@ -688,8 +715,8 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
         for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++k) {
             const K2Item item = items[it];
             const PhiloxKey key = make_key(seeds.s[item.mat - seed_base]);
-            const int sb = k % nslabs;
-            ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_empty[sb]), ((k / nslabs) & 1) ^ 1, abort);
+            const int sb = nslabs == 2 ? (k & 1) : 0;
+            ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_empty[sb]), (((nslabs == 2 ? (k >> 1) : k) & 1) ^ 1), abort);
             if (!ok) break;
             const uint32_t slab = slab0 + sb * slab_bytes;
             // the first slab (every slab, with a single buffer) is shared with the combine warps

@@ -218,22 +218,22 @@ inline void plan_compress_pair(TcSet& set, const std::vector<flora_mat>& G, int 
     if (S & (S - 1)) S = 2;
     const size_t g_stage = (size_t)T * G_TILE_BYTES, a_stage = (size_t)(N / 2) * 128, staging = 2 * (size_t)S_CHUNK_BYTES_K1;
     const size_t ring_budget = SMEM_BUDGET - sizeof(PairSmem) - 1024 - staging;
-    // A tiles are made on chip and travel between the CTAs of a cluster, whose slowest member paces all: four stages
-    // (three when that leaves fewer than three for G).  The G tiles come from HBM and get the rest.
-    int astages = 4;
-    if ((ring_budget - astages * a_stage) / g_stage < 3) astages = 3;
+    // A tiles are made on chip by warps that each need about two microseconds for their share of a slice, and travel
+    // between the CTAs of a cluster, whose slowest member paces all: six stages keep enough slices in the making
+    // (five when that leaves fewer than three stages for G).  The G tiles come from HBM and get the rest.
+    int astages = 6;
+    if ((ring_budget - astages * a_stage) / g_stage < 3) astages = 5;
     astages = tune_knob("FLORA_K1_ASTAGES", astages, 2, 8);
     int gstages = (int)std::min<size_t>(PAIR_RELAY_DEPTH - 1, (ring_budget - astages * a_stage) / g_stage);
     gstages = tune_knob("FLORA_K1_GSTAGES", std::max(1, gstages), 1, std::max(1, gstages));
-    int GW = tune_knob("FLORA_K1_GEN_WARPS", PAIR_MAX_GEN_WARPS, 4, PAIR_MAX_GEN_WARPS) & ~3;
-    // generator teams: as many as keep every thread of a team busy with at least one task per slice
+    // Worker warps claim generation work items (32 tasks of one slice) in order.  A warp waits for its stage by the
+    // parity of the stage's use count, which is only sound while no claim is a whole ring ahead of the oldest
+    // unfinished one: the warps together must hold fewer than (astages - 1) steps' worth of items.
+    int GW = tune_knob("FLORA_K1_GEN_WARPS", PAIR_MAX_GEN_WARPS, 12, PAIR_MAX_GEN_WARPS) & ~3;
     {
-        const int tile_tasks = N / S * 8;
-        int P = 1;
-        while (2 * P <= astages && GW % (2 * P) == 0 && 32 * GW / (2 * P) >= tile_tasks) P *= 2;
-        P = tune_knob("FLORA_K1_TEAMS", P, 1, 8);
-        while (P > 1 && (GW % P || P > astages || (P & (P - 1)))) --P;
-        set.P = P;
+        const int parts = (N / S * 8 + 31) / 32;
+        while (GW > 12 && (GW + PAIR_EPI_WARPS + parts - 1) / parts + 1 >= astages) GW -= 4;    // (the kernel's warp layout wants at least 12)
+        set.P = 1;
     }
     set.k1_pair = true;
     set.k1_n = N;
@@ -862,7 +862,7 @@ inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, 
         if (pair) {
             const int* slot_table = set.d_slots + set.k1_slots_begin[l];
             e = cudaLaunchKernelEx(&cfg, compress_pair_kernel, mats, items, slot_table, table, seed_base, r, set.k1_n, scale, a, b, set.gstages,
-                                   set.astages, set.S, set.GW, set.P, lw);
+                                   set.astages, set.S, set.GW, lw);
         } else {
             e = cudaLaunchKernelEx(&cfg, compress_tc_kernel, mats, items, table, seed_base, r, scale, a, b, set.T, set.gstages, set.astages, set.S,
                                    set.GW, set.P, lw);
