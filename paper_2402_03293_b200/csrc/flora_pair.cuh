@@ -75,15 +75,15 @@ compress_pair_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict
     if (threadIdx.x == 0) {
         for (int s = 0; s < gstages; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->full_g[s]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctl->empty_g[s]), 1);                    // the pair's MMAs have consumed the G tiles
+            ptx::mbar_init(ptx::smem_addr(&ctl->empty_g[s]), 2);                    // both MMA issuers of the pair have consumed the G tiles
         }
         for (int s = 0; s < astages; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->full_a[s]), 1);                     // the forwarder's arrival + the peers' bytes
             ptx::mbar_init(ptx::smem_addr(&ctl->slice_ready[s]), (uint32_t)((N / S * 8 + 31) >> 5));   // one arrival per work item of the step
-            ptx::mbar_init(ptx::smem_addr(&ctl->empty_a[s]), pairs);                // every pair of the cluster has consumed the tile
+            ptx::mbar_init(ptx::smem_addr(&ctl->empty_a[s]), 2 * pairs);            // both MMA issuers of every pair of the cluster have consumed the tile
         }
         for (int s = 0; s < PAIR_RELAY_DEPTH; ++s) ptx::mbar_init(ptx::smem_addr(&ctl->peer_full[s]), 1);
-        ptx::mbar_init(ptx::smem_addr(&ctl->acc_full), 1);
+        ptx::mbar_init(ptx::smem_addr(&ctl->acc_full), 2);
         ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty), 2 * PAIR_EPI_WARPS);        // the epilogue warps of both CTAs of the pair
         ctl->abort = 0;
         ctl->epi_go[0] = ctl->epi_go[1] = 0;
@@ -139,9 +139,14 @@ compress_pair_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict
                     ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[k % gstages]), (uint32_t)(k / gstages) & 1u, abort);
             }
         }
-    } else if (role == 1) {
-        // ------------------------------------------------------------------ MMA issuer (the pair's leader only)
+    } else if (role == 1 || (role == 3 && half == 0)) {
+        // ------------------------------------------------------------------ MMA issuers (the pair's leader only)
+        // Two threads in two warps, one per 128-row tile: a thread gets an MMA accepted only every 120 cycles or so
+        // whatever its size, and between the MMAs of two steps come its waits and commits, so one thread alone leaves
+        // the tensor core idle a third of the time.  Each commits its own MMAs to the barriers that release a stage;
+        // those barriers count both.  (The follower's warp of role 1 has nothing to do; its warp of role 3 is the relay.)
         if (lane == 0 && half == 0) {
+            const int ti = role == 1 ? 0 : 1;
             const uint32_t idesc = ptx::umma_idesc_bf16_mn(256u, (uint32_t)N);
             const uint64_t desc_base = ptx::umma_desc_k_sw128(smem_base);
             const uint16_t mask_pair = (uint16_t)(3u << rank), mask_all = (uint16_t)((1u << S) - 1u);
@@ -166,10 +171,10 @@ compress_pair_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict
                         // offsets address the follower's copy of the rings
                         const uint64_t dstage = desc_base + (uint64_t)((sg * g_bytes) >> 4);
                         const uint64_t da_tile = desc_base + (uint64_t)((a_ring - smem_base + sa * a_bytes) >> 4);
-                        for (int t = 0; t < pair_tiles; ++t) {
+                        if (ti < pair_tiles) {
 #pragma unroll
                             for (int kk = 0; kk < 4; ++kk)
-                                ptx::umma_bf16_pair(tmem + t * N, dstage + (uint64_t)((t * G_TILE_BYTES + kk * 32) >> 4), da_tile + (uint64_t)(kk * 2), idesc,
+                                ptx::umma_bf16_pair(tmem + ti * N, dstage + (uint64_t)((ti * G_TILE_BYTES + kk * 32) >> 4), da_tile + (uint64_t)(kk * 2), idesc,
                                                     (ks | kk) != 0);
                         }
                         ptx::umma_commit_pair(ebar_g, mask_pair);
@@ -217,7 +222,7 @@ compress_pair_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict
             }
         }
     } else if (role == 3) {
-        // ------------------------------------------------------------------ relay (follower only): tells the leader that this CTA's
+        // ------------------------------------------------------------------ relay (follower only; the leader's warp issues MMAs, above): tells the leader that this CTA's
         // G tiles and half of the A tile of a step are in place
         if (lane == 0 && half == 1) {
             int g = 0;
