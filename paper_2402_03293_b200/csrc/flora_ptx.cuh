@@ -105,40 +105,16 @@ __device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, uint32_t a,
 {
     asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
-// Arrive on an mbarrier of another CTA of the cluster; earlier writes of this thread are released to the cluster.
+// Arrive on an mbarrier of another CTA of the cluster.  Default semantics (release at CTA scope): what the arrival
+// announces here was written by the asynchronous proxy (TMA, bulk copies, the tensor core) and seen complete by the
+// arriving thread, not written by that thread; a release at cluster scope costs the thread most of a microsecond.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
-{
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return done != 0;
-}
-// mbar_wait with cluster-scope acquire: the arrivals come from other CTAs of the cluster.
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort)
-{
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    const unsigned long long t0 = globaltimer();
-    for (uint32_t spin = 1;; ++spin) {
-        if (mbar_try_wait_cluster(bar, parity)) return true;
-        if ((spin & 0xFF) == 0) {
-            if (*abort) return false;
-            if (globaltimer() - t0 > WAIT_LIMIT_NS) {
-                *abort = 1;
-                atomicExch(&g_flora_error_word, 1);
-                return false;
-            }
-        }
-    }
-}
+// Waits on a barrier of this CTA on which other CTAs of the cluster (or the tensor core on their behalf) arrive.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) { return mbar_try_wait(bar, parity); }
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort) { return mbar_wait(bar, parity, abort); }
 // Bulk copy from this CTA's shared memory into a peer CTA's shared memory; the bytes are counted on the
 // peer's mbarrier.  Both addresses are 16-byte aligned, the size a multiple of 16.
 __device__ __forceinline__ void bulk_copy_to_peer(uint32_t dst_cluster_addr, uint32_t src_local_addr, uint32_t bytes, uint32_t bar_cluster_addr)
