@@ -245,7 +245,7 @@ flora_status flora_transfer_axpby(flora_mat* dst, const flora_mat* src, int64_t 
     const int r = (int)dst->cols;
     if (operand == FLORA_BF16 && g_force_path.load() != 1) {
         std::vector<GramJob> jobs(1);
-        jobs[0] = GramJob{nullptr, (float*)dst->data, (const float*)src->data, dst->ld, src->ld, (int32_t)dst->rows, (int32_t)m, seed_old, seed_new};
+        jobs[0] = GramJob{nullptr, (float*)dst->data, (const float*)src->data, dst->ld, src->ld, (int32_t)dst->rows, (int32_t)m, seed_old, seed_new, 0, 0};
         if (dst->rows <= 0x7FFFFFFF && m <= 0x7FFFFFFF) return transfer_tc(jobs, r, a, b, as_stream(stream), g_launches);
     }
     float* T = nullptr;
@@ -273,7 +273,13 @@ flora_status flora_resample_transfer_static(flora_mat* M, int64_t m, int32_t ope
     float* T = nullptr;
     st = static_scratch_for_current_device(&T);
     if (st) return st;
-    // T is cleared inside (it still holds the previous call's product), then filled and applied
+    // T is cleared inside (it still holds the previous call's product), then filled and applied; bf16 operands take the
+    // tensor-core kernels of flora_resample_transfer (one matrix needs no tables: its job travels as a kernel parameter)
+    if (operand == FLORA_BF16 && g_force_path.load() != 1 && M->rows <= 0x7FFFFFFF && m <= 0x7FFFFFFF) {
+        std::vector<GramJob> jobs(1);
+        jobs[0] = GramJob{nullptr, (float*)M->data, (const float*)M->data, M->ld, M->ld, (int32_t)M->rows, (int32_t)m, seed_old, seed_new, 0, 0};
+        return transfer_tc(jobs, (int)r, 1.0f, 0.0f, as_stream(stream), g_launches, nullptr, nullptr, T);
+    }
     return transfer_with_scratch(M, M, m, operand, seed_old, seed_new, 1.0f, 0.0f, T, as_stream(stream));
 }
 
@@ -399,8 +405,8 @@ flora_status flora_set_decompress_apply(flora_set* set, const uint64_t* seeds, f
 }
 
 // dst.S[i] <- b dst.S[i] + a src[i] (A(old_i) A(new_i)^T) for every matrix of the set `dst`.
-static flora_status set_transfer(flora_set* set, const std::vector<flora_mat>& src, const uint64_t* seeds_old, const uint64_t* seeds_new, float a,
-                                 float b, void* stream)
+static flora_status set_transfer(flora_set* set, const std::vector<flora_mat>& src, const TcMatrix* src_mats, const uint64_t* seeds_old,
+                                 const uint64_t* seeds_new, float a, float b, void* stream)
 {
     if (!set || !seeds_old || !seeds_new) return FLORA_ERR_NULL;
     const std::vector<flora_mat>& big = set->has_G ? set->G : set->W;
@@ -415,9 +421,9 @@ static flora_status set_transfer(flora_set* set, const std::vector<flora_mat>& s
         for (size_t i = 0; i < set->S.size(); ++i) {
             if (set->S[i].rows == 0) continue;
             jobs.push_back(GramJob{nullptr, (float*)set->S[i].data, (const float*)src[i].data, set->S[i].ld, src[i].ld,
-                                   (int32_t)set->S[i].rows, (int32_t)big[i].cols, seeds_old[i], seeds_new[i]});
+                                   (int32_t)set->S[i].rows, (int32_t)big[i].cols, seeds_old[i], seeds_new[i], (int32_t)i, 0});
         }
-        return transfer_tc(jobs, r, a, b, as_stream(stream), g_launches);
+        return transfer_tc(jobs, r, a, b, as_stream(stream), g_launches, set->tc.d_mats, src_mats);
     }
     if (scratch_alloc((void**)&T, sizeof(float) * r * r, as_stream(stream)) != cudaSuccess) {
         cudaGetLastError();
@@ -435,7 +441,7 @@ static flora_status set_transfer(flora_set* set, const std::vector<flora_mat>& s
 flora_status flora_set_resample_transfer(flora_set* set, const uint64_t* seeds_old, const uint64_t* seeds_new, void* stream)
 {
     if (!set) return FLORA_ERR_NULL;
-    return set_transfer(set, set->S, seeds_old, seeds_new, 1.0f, 0.0f, stream);
+    return set_transfer(set, set->S, set->tc.d_mats, seeds_old, seeds_new, 1.0f, 0.0f, stream);
 }
 
 flora_status flora_set_transfer_axpby(flora_set* dst, const flora_set* src, const uint64_t* seeds_old, const uint64_t* seeds_new, float a, float b,
@@ -445,14 +451,14 @@ flora_status flora_set_transfer_axpby(flora_set* dst, const flora_set* src, cons
     if (src->S.size() != dst->S.size() || src->r != dst->r) return FLORA_ERR_SHAPE;
     for (size_t i = 0; i < dst->S.size(); ++i)
         if (src->S[i].rows != dst->S[i].rows) return FLORA_ERR_SHAPE;
-    return set_transfer(dst, src->S, seeds_old, seeds_new, a, b, stream);
+    return set_transfer(dst, src->S, src->tc.d_mats, seeds_old, seeds_new, a, b, stream);
 }
 
 flora_status flora_set_momentum_step_resampled(flora_set* set, float beta, const uint64_t* seeds_old, const uint64_t* seeds_new, void* stream)
 {
     if (!set || !seeds_old || !seeds_new) return FLORA_ERR_NULL;
     if (!set->has_G) return FLORA_ERR_UNSUPPORTED;
-    flora_status st = set_transfer(set, set->S, seeds_old, seeds_new, beta, 0.0f, stream);
+    flora_status st = set_transfer(set, set->S, set->tc.d_mats, seeds_old, seeds_new, beta, 0.0f, stream);
     if (st) return st;
     return set_compress(set, seeds_new, 1.0f - beta, 1.0f, stream);
 }

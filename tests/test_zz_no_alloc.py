@@ -15,7 +15,7 @@ import pytest
 import torch
 
 from paper_2402_03293_b200 import binding as fb
-from tests.parity_util import TOL, rel_err
+from tests.parity_util import TOL, oracle_transfer, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -33,7 +33,26 @@ def test_static_scratch_variant_matches_the_allocating_one_twice_in_a_row():
             fb.flora_resample_transfer_static(got, m, operand, s_old + rep, s_new + rep)
             torch.cuda.synchronize()
             assert rel_err(got.cpu().numpy(), ref.cpu().numpy()) <= TOL[operand], (rep, n, m, r)
+            # and against the CPU oracle, which evaluates (M A_old) A_new^T in the printed order
+            want = oracle_transfer(M0, M0, m, operand, s_old + rep, s_new + rep, 1.0, 0.0)
+            assert rel_err(got.cpu().numpy(), want) <= TOL[operand], ("oracle", rep, n, m, r)
     assert fb.flora_device_status() == 0
+
+
+def test_static_scratch_variant_leaves_device_memory_as_it_found_it():
+    # a caller whose device memory is fully planned must see the same amount of free memory before and after the
+    # call, from the driver's point of view (an allocation that was freed again into a pool would still show here)
+    dev = "cuda"
+    for n, m, r, operand in [(384, 1024, 128, "bf16"), (200, 300, 48, "f32")]:
+        M = torch.randn(n, r, device=dev)
+        fb.flora_resample_transfer_static(M, m, operand, 5, 6)      # first use of these kernels: module loading may allocate
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
+        for k in range(3):
+            fb.flora_resample_transfer_static(M, m, operand, 7 + k, 8 + k)
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after == free_before, (operand, free_before, free_after)
 
 
 def test_static_scratch_variant_rejects_what_does_not_fit():
