@@ -748,18 +748,38 @@ __global__ void scale_sketches_kernel(const TcMatrix* __restrict__ mats, const i
 }
 
 // bf16 copy of every sketch of the table, n x k_pad with zero padding (the M x K operand of the decompression
-// kernel for ranks above 64); blockIdx.y = matrix, one thread per pair of columns.
-__global__ void sketch_to_bf16_kernel(const TcMatrix* __restrict__ mats, int r, int k_pad)
+// kernel for ranks above 64); blockIdx.y = matrix.  A thread converts eight neighbouring columns of one row: two
+// 16-byte loads (the sketches that reach this kernel have 16-byte aligned rows), one 16-byte store; a block of 256
+// threads covers 2048 / k_pad rows at a time.
+__global__ void __launch_bounds__(256) sketch_to_bf16_kernel(const TcMatrix* __restrict__ mats, int r, int k_pad)
 {
     const TcMatrix* mat = mats + blockIdx.y;
-    const int half = k_pad >> 1;
-    const int64_t total = (int64_t)mat->n * half;
-    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t row = t / half;
-        const int j = (int)(t % half) * 2;
-        const float* src = mat->S + row * mat->lds;
-        const float a = j < r ? src[j] : 0.0f, b = j + 1 < r ? src[j + 1] : 0.0f;
-        reinterpret_cast<__nv_bfloat162*>(mat->Sb + row * k_pad)[j >> 1] = __floats2bfloat162_rn(a, b);
+    const int groups = k_pad >> 3;                        // 8-column groups per row: 8, 16, 24 or 32
+    const int rows_per_block = 256 / groups;
+    const int g = (int)threadIdx.x % groups, lr = (int)threadIdx.x / groups;
+    if (lr >= rows_per_block) return;
+    const int j = g * 8;
+    const float* S = mat->S;
+    const int64_t lds = mat->lds;
+    __nv_bfloat16* Sb = mat->Sb;
+    for (int row = (int)blockIdx.x * rows_per_block + lr; row < mat->n; row += (int)gridDim.x * rows_per_block) {
+        const float* src = S + (int64_t)row * lds + j;
+        float v[8];
+        if (j + 7 < r) {
+            const float4 a = *reinterpret_cast<const float4*>(src), b = *reinterpret_cast<const float4*>(src + 4);
+            v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] = j + e < r ? src[e] : 0.0f;
+        }
+        uint4 out;
+        __nv_bfloat162 p0 = __floats2bfloat162_rn(v[0], v[1]), p1 = __floats2bfloat162_rn(v[2], v[3]);
+        __nv_bfloat162 p2 = __floats2bfloat162_rn(v[4], v[5]), p3 = __floats2bfloat162_rn(v[6], v[7]);
+        out.x = *reinterpret_cast<uint32_t*>(&p0);
+        out.y = *reinterpret_cast<uint32_t*>(&p1);
+        out.z = *reinterpret_cast<uint32_t*>(&p2);
+        out.w = *reinterpret_cast<uint32_t*>(&p3);
+        *reinterpret_cast<uint4*>(Sb + (int64_t)row * k_pad + j) = out;
     }
 }
 

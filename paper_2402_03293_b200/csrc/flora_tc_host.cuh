@@ -893,7 +893,8 @@ inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float s
         const int k_pad = (r + 63) & ~63;
         int max_rows = 1;
         for (const auto& tm : set.h_mats) max_rows = std::max(max_rows, tm.n);
-        const unsigned bx = (unsigned)std::min<int64_t>(1024, ((int64_t)max_rows * (k_pad / 2) + 1023) / 1024);   // ~4 pairs per thread
+        const int rows_per_block = 256 / (k_pad / 8);
+        const unsigned bx = (unsigned)std::max<int64_t>(1, std::min<int64_t>(256, ((int64_t)max_rows + 4 * rows_per_block - 1) / (4 * rows_per_block)));   // about four rows per thread
         for (int begin = 0; begin < set.count; begin += 65535) {
             dim3 grid(bx, (unsigned)std::min(65535, set.count - begin));
             sketch_to_bf16_kernel<<<grid, 256, 0, st>>>(set.d_mats + begin, r, k_pad);
