@@ -402,7 +402,7 @@ def run_flora(args):
         barrier()
         blocks.append(e0.elapsed_time(e1))
         spent += blocks[-1] * 1e-3
-        done = spent >= MIN_TIMED_SECONDS or len(blocks) >= 200
+        done = spent >= args.min_seconds or len(blocks) >= 200
         if dist:                        # all ranks stop together
             flag = torch.tensor([1.0 if done else 0.0], device=dev)
             dist.all_reduce(flag, op=dist.ReduceOp.MAX)
@@ -520,6 +520,8 @@ def main():
     ap.add_argument("--impl", default="flora", choices=["flora", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=[n for n in wl.CONFIG_ORDER if wl.WORKLOADS[n].dtype == "bf16"])
     ap.add_argument("--rank", type=int, default=0, help="rank r of the sketches (default: the workload's)")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
+                    help="repeat the block of --steps steps until this much device time has been measured (0: one block, e.g. under a profiler)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "flora" else args.warmup
     if args.impl == "reference":

@@ -198,6 +198,17 @@ flora_status flora_set_compress_accumulate_from_host(flora_set* set, const void*
 flora_status flora_set_read_weights_to_host(flora_set* set, void* const* host_W, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Reproducibility.
+ * ------------------------------------------------------------------------------------------- */
+/* A is a function of (seed, j, k) alone, so every result is reproducible up to the order of floating-point
+ * additions.  By default the work of one matrix may be split over CTAs that add their partial sums in arrival
+ * order (compression over column ranges of a wide matrix; the r x r product of the transfer over column ranges),
+ * which can change the last bits from run to run.  on != 0: sets created from now on give every row of a sketch a
+ * single owner, and every transfer from now on sums its r x r product in one CTA per matrix, so that repeated runs
+ * on the same inputs are bit-identical (slower on few, wide matrices).  Process-wide; default off. */
+void flora_set_deterministic(int on);
+
+/* ---------------------------------------------------------------------------------------------
  * Diagnostics.
  * ------------------------------------------------------------------------------------------- */
 /* Test hook: 0 = choose the kernel automatically (tensor-core kernels when dtype, alignment and

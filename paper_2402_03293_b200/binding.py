@@ -29,7 +29,7 @@ EXPORTS = [
     "flora_set_rebind_gradients", "flora_set_compress_accumulate", "flora_set_momentum_step",
     "flora_set_decompress_apply", "flora_set_resample_transfer", "flora_set_transfer_axpby", "flora_set_momentum_step_resampled", "flora_set_zero_state", "flora_derive_seed",
     "flora_resamples_at", "flora_set_upload_gradients", "flora_set_compress_accumulate_from_host", "flora_set_read_weights_to_host",
-    "flora_debug_force_path", "flora_debug_plan", "flora_debug_wait_timeout_selftest", "flora_launch_count", "flora_device_status", "flora_status_string", "flora_version",
+    "flora_debug_force_path", "flora_set_deterministic", "flora_debug_plan", "flora_debug_wait_timeout_selftest", "flora_launch_count", "flora_device_status", "flora_status_string", "flora_version",
 ]
 
 
@@ -81,6 +81,7 @@ def load() -> ctypes.CDLL:
             "flora_set_read_weights_to_host": (I32, [P, ctypes.POINTER(P), P]),
             "flora_set_upload_gradients": (I32, [P, ctypes.POINTER(P), P]),
             "flora_debug_force_path": (None, [ctypes.c_int]),
+            "flora_set_deterministic": (None, [ctypes.c_int]),
             "flora_debug_plan": (I32, [P, P, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, P, ctypes.c_int64, P, P]),
             "flora_debug_wait_timeout_selftest": (I32, [P]),
             "flora_launch_count": (U64, []),
@@ -201,6 +202,10 @@ def flora_resamples_at(t: int, kappa: int) -> bool:
 
 def flora_debug_force_path(path: int) -> None:
     load().flora_debug_force_path(path)
+
+
+def flora_set_deterministic(on: bool) -> None:
+    load().flora_set_deterministic(1 if on else 0)
 
 
 def flora_debug_plan(shapes, r: int, which: str):

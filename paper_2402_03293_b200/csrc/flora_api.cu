@@ -539,6 +539,8 @@ int flora_resamples_at(int64_t t, int64_t kappa) { return (kappa > 0 && t >= 0 &
 // ------------------------------------------------------------------------------------------------
 void flora_debug_force_path(int path) { g_force_path.store(path == 1 ? 1 : 0); }
 
+void flora_set_deterministic(int on) { deterministic_flag().store(on ? 1 : 0); }
+
 flora_status flora_debug_plan(const int64_t* rows, const int64_t* cols, int64_t count, int32_t r, int32_t which, int32_t* items, int64_t capacity,
                               int64_t* n_items, int32_t* params)
 {

@@ -677,7 +677,9 @@ inline flora_status transfer_tc(std::vector<GramJob>& jobs, int r, float a, floa
     for (const auto& j : jobs) total_steps += (j.m + kw - 1) / kw;
     const bool single = jobs.size() == 1;
     // a single matrix: one wave of equal chunks; a set: about three items per SM, the largest first
-    const int64_t chunk = std::max<int64_t>(1, single ? (total_steps + sms - 1) / sms : (total_steps + 3 * sms - 1) / (3 * sms));
+    // (deterministic mode: one CTA per matrix, so that its r x r product is summed in one fixed order)
+    const int64_t chunk = deterministic_flag().load() ? std::max<int64_t>(1, total_steps)
+                          : std::max<int64_t>(1, single ? (total_steps + sms - 1) / sms : (total_steps + 3 * sms - 1) / (3 * sms));
     const size_t t_bytes = (((size_t)r * r * sizeof(float)) + 255) & ~(size_t)255;
     const int r_m = (r + 127) & ~127, r_n = (r + 15) & ~15;
     const size_t smem = 2 * (size_t)(r_m + r_n) * 128 + sizeof(GramSmem) + 1024;

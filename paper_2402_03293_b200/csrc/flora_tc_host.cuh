@@ -127,6 +127,14 @@ inline int sm_count()
 
 constexpr size_t SMEM_BUDGET = 226 * 1024;   // per SM, below the 227 KB limit of sm_100
 
+// Process-wide switch (flora_set_deterministic): when on, no sum is split over CTAs that add their parts in arrival
+// order, so that repeated runs give the same bits.  Read when a set is planned and at every transfer.
+inline std::atomic<int>& deterministic_flag()
+{
+    static std::atomic<int> flag{0};
+    return flag;
+}
+
 // Tile shapes and the work split are chosen by the planners below.  A build with -DFLORA_TUNE lets environment
 // variables override single choices for parameter sweeps (they never change what is computed); the library as
 // shipped reads no environment variable.
@@ -308,7 +316,7 @@ inline void plan_compress_pair(TcSet& set, const std::vector<flora_mat>& G, int 
     // a schedule without any split over columns is preferred when it is nearly as short: every row of a sketch then
     // has one owner, so a momentum update needs neither the pre-scaling pass nor atomic adds
     build_units((int64_t)1 << 60, cand_units, cand_split);
-    if (assign(cand_units, 0, cand_units.size(), nullptr) <= 1.12 * best_span) {
+    if (deterministic_flag().load() || assign(cand_units, 0, cand_units.size(), nullptr) <= 1.12 * best_span) {
         units = cand_units;
         set.split_mats = cand_split;
     }
@@ -505,7 +513,7 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
     // has one owner, so a momentum update needs neither the pre-scaling pass nor atomic adds
     if (!fixed_waves) {
         build_units((int64_t)1 << 60, cand_units, cand_split);
-        if (makespan(cand_units) <= 1.12 * best_span) {
+        if (deterministic_flag().load() || makespan(cand_units) <= 1.12 * best_span) {
             units = cand_units;
             set.split_mats = cand_split;
         }
