@@ -26,7 +26,14 @@
  *  - The rank r is the column count of the sketch, 1 <= r <= 256.
  *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *    Calls are asynchronous: they enqueue work on `stream` and return; they
- *    never synchronise the device.
+ *    do not synchronise the device.  One exception: the first single-matrix
+ *    call that meets a new (operation, addresses, shape, rank) on the
+ *    tensor-core path builds its plan (work split, TMA descriptors, a few KB
+ *    of device tables, for ranks above 64 a bf16 copy of the sketch for the
+ *    decompression) with a device allocation and a synchronisation of
+ *    `stream`; the 32 most recent plans are kept, so a training loop pays
+ *    this once per matrix.  flora_set_* calls never do: a set is planned
+ *    when it is created.
  *  - Errors are reported by the returned status only; arguments are checked
  *    before anything is launched, and a failed check launches nothing.
  *  - A[j,k] depends on (seed, j, k) only and on r only through the factor

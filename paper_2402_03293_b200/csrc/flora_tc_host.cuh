@@ -12,6 +12,7 @@
 #include <vector>
 
 #include <mutex>
+#include <new>
 
 #include "flora_pair.cuh"
 #include "flora_pool.cuh"
@@ -881,15 +882,91 @@ inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, 
     return cudaPeekAtLastError() == cudaSuccess ? FLORA_OK : FLORA_ERR_CUDA;
 }
 
+// Single-matrix calls go through a set of one matrix.  Planning it (work split, tensor maps, device tables) costs far
+// more than the launch, and an optimizer calls with the same matrices step after step: the most recent plans are kept,
+// keyed by device, operation, addresses, shapes and rank.  A plan only names addresses and shapes, so it stays valid
+// when the caller's buffers are rewritten (or freed and handed out again with the same shape).  Calls that use the
+// cache are serialised by its mutex; a plan is built with a synchronous upload, so any stream may use it afterwards.
+struct SinglePlanKey {
+    int dev, kind, r, det;
+    const void *big, *sketch;
+    int64_t rows, cols, ld, lds;
+    bool operator==(const SinglePlanKey& o) const
+    {
+        return dev == o.dev && kind == o.kind && r == o.r && det == o.det && big == o.big && sketch == o.sketch && rows == o.rows &&
+               cols == o.cols && ld == o.ld && lds == o.lds;
+    }
+};
+struct SinglePlan {
+    SinglePlanKey key;
+    TcSet set;
+};
+constexpr size_t SINGLE_PLAN_CACHE = 32;
+inline std::mutex& single_plan_mutex()
+{
+    static std::mutex m;
+    return m;
+}
+// Call with single_plan_mutex() held.  kind 0: compression (big = G), 1: decompression (big = W).
+inline TcSet* single_plan(int kind, const flora_mat& big, const flora_mat& sketch, cudaStream_t st, flora_status* rc)
+{
+    static std::vector<SinglePlan*> cache;                     // most recently used first
+    *rc = FLORA_OK;
+    SinglePlanKey key;
+    memset(&key, 0, sizeof(key));
+    if (cudaGetDevice(&key.dev) != cudaSuccess) {
+        cudaGetLastError();
+        *rc = FLORA_ERR_CUDA;
+        return nullptr;
+    }
+    key.kind = kind;
+    key.r = (int)sketch.cols;
+    key.det = deterministic_flag().load();
+    key.big = big.data;
+    key.sketch = sketch.data;
+    key.rows = big.rows;
+    key.cols = big.cols;
+    key.ld = big.ld;
+    key.lds = sketch.ld;
+    for (size_t i = 0; i < cache.size(); ++i)
+        if (cache[i]->key == key) {
+            SinglePlan* hit = cache[i];
+            cache.erase(cache.begin() + i);
+            cache.insert(cache.begin(), hit);
+            return &hit->set;
+        }
+    SinglePlan* plan = new (std::nothrow) SinglePlan();
+    if (!plan) {
+        *rc = FLORA_ERR_ALLOC;
+        return nullptr;
+    }
+    plan->key = key;
+    std::vector<flora_mat> b(1, big), s(1, sketch), none;
+    *rc = kind == 0 ? tc_set_build_on(plan->set, b, none, s, false, st) : tc_set_build_on(plan->set, none, b, s, false, st);
+    if (*rc == FLORA_OK && cudaStreamSynchronize(st) != cudaSuccess) *rc = FLORA_ERR_CUDA;      // the tables are in place for every stream
+    if (*rc != FLORA_OK) {
+        tc_set_free(plan->set);
+        delete plan;
+        return nullptr;
+    }
+    cache.insert(cache.begin(), plan);
+    if (cache.size() > SINGLE_PLAN_CACHE) {
+        SinglePlan* old = cache.back();
+        cache.pop_back();
+        tc_set_free(old->set);                                 // cudaFree waits for kernels that still read the tables
+        delete old;
+    }
+    return &plan->set;
+}
+
 inline flora_status tc_compress_single(const flora_mat* G, flora_mat* S, uint64_t seed, float a, float b, cudaStream_t st,
                                        std::atomic<uint64_t>& launches)
 {
-    TcSet set;
-    std::vector<flora_mat> g(1, *G), s(1, *S), none;
-    flora_status rc = tc_set_build_on(set, g, none, s, true, st);
-    if (rc == FLORA_OK) rc = set.compress_ready ? tc_set_compress(set, &seed, a, b, st, launches) : FLORA_ERR_UNSUPPORTED;
-    tc_set_free_stream(set, st);
-    return rc;
+    std::lock_guard<std::mutex> lock(single_plan_mutex());
+    flora_status rc;
+    TcSet* set = single_plan(0, *G, *S, st, &rc);
+    if (!set) return rc;
+    return set->compress_ready ? tc_set_compress(*set, &seed, a, b, st, launches) : FLORA_ERR_UNSUPPORTED;
 }
 
 inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float step, cudaStream_t st,
@@ -931,12 +1008,11 @@ inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float s
 inline flora_status tc_decompress_single(flora_mat* W, const flora_mat* S, uint64_t seed, float step, cudaStream_t st,
                                          std::atomic<uint64_t>& launches)
 {
-    TcSet set;
-    std::vector<flora_mat> w(1, *W), s(1, *S), none;
-    flora_status rc = tc_set_build_on(set, none, w, s, true, st);
-    if (rc == FLORA_OK) rc = set.decompress_ready ? tc_set_decompress(set, &seed, step, st, launches) : FLORA_ERR_UNSUPPORTED;
-    tc_set_free_stream(set, st);
-    return rc;
+    std::lock_guard<std::mutex> lock(single_plan_mutex());
+    flora_status rc;
+    TcSet* set = single_plan(1, *W, *S, st, &rc);
+    if (!set) return rc;
+    return set->decompress_ready ? tc_set_decompress(*set, &seed, step, st, launches) : FLORA_ERR_UNSUPPORTED;
 }
 
 inline bool tc_decompress_supported(const flora_mat* big, const flora_mat* sketch)
