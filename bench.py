@@ -193,7 +193,7 @@ class Rotating:
         self.sets[0].zero_state(stream)
 
 
-def make_stepper(w: wl.Workload, acc: Rotating, mom, count: int, base_seed: int):
+def make_stepper(w: wl.Workload, acc: Rotating, mom, count: int, base_seed: int, exchange=None):
     """One Flora step of the workload's mode as a closure, sequenced by the host classes of Algorithms 1 and 2."""
     if w.mode == "accumulate":
         cyc = hostlogic.AccumulationCycle(acc, count, w.tau, base_seed)
@@ -201,6 +201,8 @@ def make_stepper(w: wl.Workload, acc: Rotating, mom, count: int, base_seed: int)
         def step():
             for _ in range(w.tau):
                 cyc.accumulate()
+            if exchange:
+                exchange()
             cyc.apply(LR)
         return step, f"{w.tau} x compress_accumulate + decompress_apply + zero C"
     if w.mode == "momentum":
@@ -222,6 +224,8 @@ def make_stepper(w: wl.Workload, acc: Rotating, mom, count: int, base_seed: int)
     def step():
         for _ in range(w.tau):
             both.accumulate()
+        if exchange:
+            exchange()
         both.apply(LR)
     return step, (f"{w.tau} x compress_accumulate into C + transfer_axpby (M <- beta M + (1-beta)/tau C A_acc A_mom^T) + "
                   f"decompress_apply of M + zero C; M resampled every {w.kappa} steps")
@@ -365,7 +369,14 @@ def run_flora(args):
     mset = fb.FloraSet(None, W, M) if both else None
     acc = Rotating(sets)
     mom = Rotating([mset]) if both else None
-    step, what = make_stepper(w, acc, mom, count, base_seed=17 + rank)
+    # --exchange sketches (N > 1, accumulation workloads): the ranks are data-parallel workers that hold different
+    # micro-batches and the same seeds; they sum their sketches C over NCCL before the update (linearity, Section 2.2)
+    exchange = None
+    if args.exchange == "sketches" and dist and w.mode != "momentum":
+        exchange = lambda: replicas.allreduce_sketches(C, dist)
+    step, what = make_stepper(w, acc, mom, count, base_seed=17 + (0 if exchange else rank), exchange=exchange)
+    if exchange:
+        what += "; sketches summed over ranks (all-reduce of C) before the update"
 
     def begin_marks():
         for rot in (acc, mom):
@@ -499,7 +510,7 @@ def run_flora(args):
                        "step": what,
                        "l2": f"inputs larger than L2: {n_sets} rotating gradient sets of {grad_set_bytes / 1e9:.2f} GB, a different one per compression",
                        "timed": f"{len(blocks)} block(s) of {args.steps} steps, {spent:.2f} s of device time; value is the median block",
-                       "multi_gpu": "independent replicas, no collective"},
+                       "multi_gpu": "data-parallel ranks, all-reduce of the sketches" if exchange else "independent replicas, no collective"},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches_per_block), "clocks": clocks,
             "ms_x_mhz_per_step": (ms / args.steps) * clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None,
         }
@@ -520,6 +531,8 @@ def main():
     ap.add_argument("--impl", default="flora", choices=["flora", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=[n for n in wl.CONFIG_ORDER if wl.WORKLOADS[n].dtype == "bf16"])
     ap.add_argument("--rank", type=int, default=0, help="rank r of the sketches (default: the workload's)")
+    ap.add_argument("--exchange", default="none", choices=["none", "sketches"],
+                    help="N > 1 only: none = independent replicas (default); sketches = data-parallel ranks that all-reduce C")
     ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
                     help="repeat the block of --steps steps until this much device time has been measured (0: one block, e.g. under a profiler)")
     args = ap.parse_args()

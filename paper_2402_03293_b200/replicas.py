@@ -25,3 +25,37 @@ def aggregate_throughput(bytes_per_rank: float, steps: int, ms_this_rank: float,
     ms = max_over_ranks(ms_this_rank, dist, device)
     return {"world": world, "ms": ms, "ms_per_step": ms / steps,
             "gbs": world * bytes_per_rank * steps / (ms * 1e-3) / 1e9}
+
+
+def allreduce_sketches(sketches, dist=None, bucket_bytes: int = 256 << 20) -> None:
+    """Data-parallel exchange step: sums the n x r sketches of all ranks in place (every rank gets the sum).
+
+    Compression is linear in the gradient (C(G1 + G2) = C(G1) + C(G2) for one projection, Section 2.2), so ranks that
+    hold different micro-batches and the same seeds can exchange their sketches instead of their n x m gradients:
+    m / r times fewer bytes on the wire.  The sketches travel in buckets of at most `bucket_bytes` (one collective
+    each), through whatever backend the process group has (NCCL between GPUs, gloo on CPU).  Identity without a
+    process group.  This is plumbing around the library's calls, not part of them: the sum over ranks is the
+    collective's, every rank then runs the same decompress-apply."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return
+    group, size = [], 0
+
+    def flush():
+        nonlocal group, size
+        if not group:
+            return
+        flat = torch.cat([s.reshape(-1) for s in group])
+        dist.all_reduce(flat, op=dist.ReduceOp.SUM)
+        offset = 0
+        for s in group:
+            s.copy_(flat[offset:offset + s.numel()].view_as(s))
+            offset += s.numel()
+        group, size = [], 0
+
+    for s in sketches:
+        nbytes = s.numel() * s.element_size()
+        if group and size + nbytes > bucket_bytes:
+            flush()
+        group.append(s)
+        size += nbytes
+    flush()
