@@ -33,7 +33,7 @@ constexpr int PAIR_RELAY_DEPTH = 8;         // ring of the follower -> leader "s
 inline int pair_threads(int gen_warps) { return 32 * (PAIR_FIXED_WARPS + gen_warps + PAIR_EPI_WARPS); }
 
 struct PairSmem {
-    uint64_t full_g[8], empty_g[8], full_a[8], slice_ready[8], empty_a[8], peer_full[PAIR_RELAY_DEPTH], acc_full, acc_empty;
+    uint64_t full_g[8], empty_g[8], full_a[8], slice_ready[8], empty_a[8], ready[PAIR_RELAY_DEPTH], acc_full, acc_empty;
     uint32_t tmem_base;
     int abort;
     int epi_go[2];
@@ -82,7 +82,10 @@ compress_pair_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict
             ptx::mbar_init(ptx::smem_addr(&ctl->slice_ready[s]), (uint32_t)((N / S * 8 + 31) >> 5));   // one arrival per work item of the step
             ptx::mbar_init(ptx::smem_addr(&ctl->empty_a[s]), 2 * pairs);            // both MMA issuers of every pair of the cluster have consumed the tile
         }
-        for (int s = 0; s < PAIR_RELAY_DEPTH; ++s) ptx::mbar_init(ptx::smem_addr(&ctl->peer_full[s]), 1);
+        // leaders: one barrier per step for all that the step's MMAs need: this CTA's G tiles (the producer's arrival and
+        // their bytes), its half of the A tile (the forwarder's arrival and the peers' bytes) and the follower's word
+        // that its own tiles are in place
+        for (int s = 0; s < PAIR_RELAY_DEPTH; ++s) ptx::mbar_init(ptx::smem_addr(&ctl->ready[s]), 3);
         ptx::mbar_init(ptx::smem_addr(&ctl->acc_full), 2);
         ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty), 2 * PAIR_EPI_WARPS);        // the epilogue warps of both CTAs of the pair
         ctl->abort = 0;
@@ -112,17 +115,18 @@ compress_pair_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict
         // ------------------------------------------------------------------ TMA producer: this CTA's rows of G
         if (lane == 0) {
             int g = 0, issued = 0;
-            RingPos pg;
+            RingPos pg, pp;
             bool ok = true;
             for (int u = u_begin; u < u_end && ok; ++u) {
                 const K1Item item = items[(size_t)u * S + rank];
                 const TcMatrix* mat = mats + item.mat;
                 if (item.tiles > 0) ptx::prefetch_tensormap(&mat->map_g);
-                for (int ks = 0; ks < item.ksteps; ++ks, ++g, pg.advance(gstages)) {
+                for (int ks = 0; ks < item.ksteps; ++ks, ++g, pg.advance(gstages), pp.advance(PAIR_RELAY_DEPTH)) {
                     const int s = pg.s;
                     ok = ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->empty_g[s]), (pg.wraps & 1u) ^ 1u, abort);
                     if (!ok) break;
-                    const uint32_t bar = ptx::smem_addr(&ctl->full_g[s]);
+                    // a leader's loads complete on the step's barrier, a follower's on its own (its relay watches that one)
+                    const uint32_t bar = half == 0 ? ptx::smem_addr(&ctl->ready[pp.s]) : ptx::smem_addr(&ctl->full_g[s]);
                     if (item.tiles > 0) {
                         ptx::mbar_arrive_expect_tx(bar, (uint32_t)item.tiles * G_TILE_BYTES);
                         for (int t = 0; t < item.tiles; ++t)
@@ -133,8 +137,10 @@ compress_pair_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict
                     issued = g + 1;
                 }
             }
-            if (*abort) {
-                // nobody consumes any more: wait (bounded) until the copies still in flight have landed
+            if (*abort && half == 1) {
+                // nobody consumes any more: wait (bounded) until the copies still in flight have landed (a leader's loads
+                // complete on barriers that also need the forwarder and the follower; after an abort the kernel's final
+                // cluster-wide barrier comes long after the two microseconds a load takes)
                 for (int k = max(0, issued - gstages); k < issued; ++k)
                     ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[k % gstages]), (uint32_t)(k / gstages) & 1u, abort);
             }
@@ -160,9 +166,7 @@ compress_pair_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict
                 if (done > 0) ok = ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->acc_empty), (uint32_t)(done - 1) & 1u, abort);
                 for (int ks = 0; ks < item.ksteps && ok; ++ks, ++g, pg.advance(gstages), pa.advance(astages), pp.advance(PAIR_RELAY_DEPTH)) {
                     const int sg = pg.s, sa = pa.s, sp = pp.s;
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[sg]), pg.wraps & 1u, abort) &&
-                         ptx::mbar_wait(ptx::smem_addr(&ctl->full_a[sa]), pa.wraps & 1u, abort) &&
-                         ptx::mbar_wait(ptx::smem_addr(&ctl->peer_full[sp]), pp.wraps & 1u, abort);
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->ready[sp]), pp.wraps & 1u, abort);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
                     const uint32_t ebar_g = ptx::smem_addr(&ctl->empty_g[sg]), ebar_a = ptx::smem_addr(&ctl->empty_a[sa]);
@@ -201,15 +205,16 @@ compress_pair_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict
         if (lane == 0) {
             const uint32_t slice_bytes = (uint32_t)(N / S) * 128u;
             int g = 0;
-            RingPos pa;
+            RingPos pa, pp;
             bool ok = true;
             for (int u = u_begin; u < u_end && ok; ++u) {
                 const int ksteps = items[(size_t)u * S + rank].ksteps;
-                for (int ks = 0; ks < ksteps; ++ks, ++g, pa.advance(astages)) {
+                for (int ks = 0; ks < ksteps; ++ks, ++g, pa.advance(astages), pp.advance(PAIR_RELAY_DEPTH)) {
                     const int s = pa.s;
                     ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slice_ready[s]), pa.wraps & 1u, abort);
                     if (!ok) break;
-                    const uint32_t fbar = ptx::smem_addr(&ctl->full_a[s]);
+                    // the same barrier offset in every CTA of this parity: the step's barrier among leaders, the A stage's among followers
+                    const uint32_t fbar = half == 0 ? ptx::smem_addr(&ctl->ready[pp.s]) : ptx::smem_addr(&ctl->full_a[s]);
                     if (pairs > 1) {
                         const uint32_t src = a_ring + s * a_bytes + pair * slice_bytes;
                         ptx::mbar_arrive_expect_tx(fbar, (uint32_t)(pairs - 1) * slice_bytes);   // own slice is in place; the peers' bytes to come
@@ -234,7 +239,7 @@ compress_pair_kernel(const TcMatrix* __restrict__ mats, const K1Item* __restrict
                     ok = ptx::mbar_wait(ptx::smem_addr(&ctl->full_g[pg.s]), pg.wraps & 1u, abort) &&
                          ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->full_a[pa.s]), pa.wraps & 1u, abort);
                     if (!ok) break;
-                    ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_addr(&ctl->peer_full[pp.s]), rank - 1));
+                    ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_addr(&ctl->ready[pp.s]), rank - 1));
                 }
             }
         } else if (lane == 0) {
