@@ -43,8 +43,8 @@ struct GramItem {           // one CTA of the gram kernel
     int32_t pad;
 };
 
-constexpr int GRAM_GEN_WARPS = 12;
-constexpr int GRAM_THREADS = 32 * (1 + GRAM_GEN_WARPS);   // warp 0: MMA issuer, warps 1..12: generators (1-4 also read back)
+constexpr int GRAM_GEN_WARPS = 20;
+constexpr int GRAM_THREADS = 32 * (1 + GRAM_GEN_WARPS);   // warp 0: MMA issuer, warps 1..20: generators (1-4 also read back)
 
 struct GramSmem {
     uint64_t full[2], empty[2], acc_full;
