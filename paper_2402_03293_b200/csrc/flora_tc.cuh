@@ -783,13 +783,22 @@ __global__ void __launch_bounds__(256) sketch_to_bf16_kernel(const TcMatrix* __r
     }
 }
 
-// S <- 0 for every matrix of the table (start of an accumulation cycle); blockIdx.y = matrix.
+// S <- 0 for every matrix of the table (start of an accumulation cycle); blockIdx.y = matrix.  Densely stored sketches
+// with 16-byte aligned storage are cleared with 16-byte stores, others element by element along each row.
 __global__ void zero_sketches_kernel(const TcMatrix* __restrict__ mats, int r)
 {
     const TcMatrix* mat = mats + blockIdx.y;
+    float* S = mat->S;
     const int64_t total = (int64_t)mat->n * r;
-    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x)
-        mat->S[(t / r) * mat->lds + (t % r)] = 0.0f;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, nthreads = (int64_t)gridDim.x * blockDim.x;
+    if (mat->lds == r && (reinterpret_cast<uintptr_t>(S) & 15) == 0) {
+        float4* S4 = reinterpret_cast<float4*>(S);
+        for (int64_t t = tid; t < (total >> 2); t += nthreads) S4[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int64_t t = (total & ~(int64_t)3) + tid; t < total; t += nthreads) S[t] = 0.0f;
+    } else {
+        for (int64_t row = blockIdx.x; row < mat->n; row += gridDim.x)
+            for (int j = (int)threadIdx.x; j < r; j += (int)blockDim.x) S[row * mat->lds + j] = 0.0f;
+    }
 }
 
 // Self-test of the bounded waits: one CTA waits on a barrier that nothing ever arrives on, with a one-millisecond
