@@ -255,10 +255,19 @@ def _mat_array(ts: Optional[Sequence[torch.Tensor]]):
     return arr
 
 
+class SeedList(list):
+    """A list of seeds that remembers its marshalled form, so that handing the same list to many calls costs nothing."""
+    _marshalled = None
+
+
 def _u64_array(vals):
     """Host array of 64-bit seeds; an array made by an earlier call is passed through unchanged."""
     if isinstance(vals, ctypes.Array):
         return vals
+    if isinstance(vals, SeedList):
+        if vals._marshalled is None or len(vals._marshalled) != len(vals):
+            vals._marshalled = (ctypes.c_uint64 * len(vals))(*[int(v) & 0xFFFFFFFFFFFFFFFF for v in vals])
+        return vals._marshalled
     return (ctypes.c_uint64 * len(vals))(*[int(v) & 0xFFFFFFFFFFFFFFFF for v in vals])
 
 

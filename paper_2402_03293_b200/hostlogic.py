@@ -11,6 +11,15 @@ from typing import List
 from . import binding
 
 
+def _derived(cache: dict, base_seed: int, count: int, epoch: int):
+    """The seeds of one epoch, derived once (they are asked for at every micro-step)."""
+    if epoch not in cache:
+        if len(cache) > 4:
+            cache.clear()
+        cache[epoch] = binding.SeedList(binding.flora_derive_seed(base_seed, i, epoch) for i in range(count))
+    return cache[epoch]
+
+
 class AccumulationCycle:
     """Algorithm 1: tau compressions into C with one projection per matrix, then one decompression
     with scale 1/tau; after that C is zeroed and the projection resampled (Section 2.4)."""
@@ -21,9 +30,10 @@ class AccumulationCycle:
         self.ops, self.count, self.tau, self.base_seed = ops, count, tau, base_seed
         self.epoch = 0
         self.micro_step = 0
+        self._seeds = {}
 
     def seeds(self) -> List[int]:
-        return [binding.flora_derive_seed(self.base_seed, i, self.epoch) for i in range(self.count)]
+        return _derived(self._seeds, self.base_seed, self.count, self.epoch)
 
     def accumulate(self, stream=None) -> bool:
         """Compress the gradients currently bound to the set; True when the cycle is full."""
@@ -54,9 +64,10 @@ class MomentumState:
         self.epoch = 0
         self.skip0 = skip_transfer_of_zero_state
         self.fuse = fuse_transfer                        # transfer and update of a resampling step as one call
+        self._seeds = {}
 
     def seeds(self, epoch: int) -> List[int]:
-        return [binding.flora_derive_seed(self.base_seed, i, epoch) for i in range(self.count)]
+        return _derived(self._seeds, self.base_seed, self.count, epoch)
 
     def step(self, lr: float, stream=None) -> None:
         fused = False
@@ -95,12 +106,13 @@ class AccumulatedMomentum:
         self.micro_step = 0
         self.acc_epoch = 0
         self.mom_epoch = 0
+        self._acc, self._mom = {}, {}
 
     def acc_seeds(self) -> List[int]:
-        return [binding.flora_derive_seed(self.base_seed, i, self.acc_epoch) for i in range(self.count)]
+        return _derived(self._acc, self.base_seed, self.count, self.acc_epoch)
 
     def mom_seeds(self, epoch: int) -> List[int]:
-        return [binding.flora_derive_seed(self.base_seed ^ 0x5DEECE66D, i, epoch) for i in range(self.count)]
+        return _derived(self._mom, self.base_seed ^ 0x5DEECE66D, self.count, epoch)
 
     def accumulate(self, stream=None) -> bool:
         """Compress the gradients currently bound to `acc`; True when the cycle is full."""
