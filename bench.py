@@ -40,8 +40,11 @@ FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1400.0
 NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
 MIN_TIMED_SECONDS = 1.5        # the K-step block is repeated until this much device time has been measured
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised
-# under profiles/ (absent = not captured since the kernel last changed)
-NCU_TRAFFIC = {}
+# under profiles/ (absent = not captured since the kernel last changed).  The benchmark's weight set is too large for a
+# multi-pass capture: the compression figure is the capture of the same kernel on one 4096 x 11008 matrix at r = 256
+# (99.5 MB for 98.6 MB algorithmic, profiles/compress_pair_kernel_single_bf16_4096x11008_r256.md), scaled by the
+# algorithmic bytes of this workload (traffic grows with the elements streamed: G is read once, C read and written once).
+NCU_TRAFFIC = {("gpt2_xl_set", 256, "compress"): int(4050124800 * 99.52 / 98.57)}
 
 
 # ------------------------------------------------------------------------------------------ helpers
