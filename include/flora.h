@@ -34,6 +34,11 @@
  *    `stream`; the 32 most recent plans are kept, so a training loop pays
  *    this once per matrix.  flora_set_* calls never do: a set is planned
  *    when it is created.
+ *  - Stream capture: the set-level transfers (flora_set_resample_transfer,
+ *    flora_set_transfer_axpby, flora_set_momentum_step_resampled),
+ *    flora_set_rebind_gradients and a single-matrix call that plans upload
+ *    small tables from ordinary host memory that the call does not keep;
+ *    do not record these into a CUDA graph.
  *  - Errors are reported by the returned status only; arguments are checked
  *    before anything is launched, and a failed check launches nothing.
  *  - A[j,k] depends on (seed, j, k) only and on r only through the factor

@@ -788,11 +788,9 @@ inline flora_status transfer_tc(std::vector<GramJob>& jobs, int r, float a, floa
         return e == cudaSuccess;
     };
     if (tiled)
-        ok = ok && (single ? cudaFuncSetAttribute(apply_gram_jobs_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apply_smem_bytes(r))
-                           : cudaFuncSetAttribute(apply_gram_jobs_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apply_smem_bytes(r))) ==
-                       cudaSuccess;
+        ok = ok && (single ? raise_smem_limit<apply_gram_jobs_kernel<true>>() : raise_smem_limit<apply_gram_jobs_kernel<false>>());
     if (single) {
-        ok = ok && cudaFuncSetAttribute(gram_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess;
+        ok = ok && raise_smem_limit<gram_tc_kernel<true>>();
         if (ok) {
             const int ks = (jobs[0].m + kw - 1) / kw;
             if (ks > 0) {
@@ -812,7 +810,7 @@ inline flora_status transfer_tc(std::vector<GramJob>& jobs, int r, float a, floa
         memcpy(tables.data(), jobs.data(), jobs.size() * sizeof(GramJob));
         // pageable source: staged by the runtime before the call returns
         ok = ok && cudaMemcpyAsync(buf + tables_off, tables.data(), tables.size(), cudaMemcpyHostToDevice, st) == cudaSuccess &&
-             cudaFuncSetAttribute(gram_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess;
+             raise_smem_limit<gram_tc_kernel<false>>();
         if (ok) {
             const GramJob* d_jobs = reinterpret_cast<const GramJob*>(buf + tables_off);
             const GramItem* d_items = reinterpret_cast<const GramItem*>(buf + tables_off + jobs_bytes);

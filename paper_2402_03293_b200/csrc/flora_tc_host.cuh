@@ -201,6 +201,17 @@ inline int resident_clusters(int S, int threads, size_t smem)
 // Cost model of the compression planners, in units of one 64-column step of a full CTA: what a work unit costs
 // before its first and after its last step (barriers, first loads, writing the accumulators out).
 constexpr double K1_UNIT_OVERHEAD_STEPS = 6.0;
+// Cost model of the r <= 64 compression planner: generating one value of A costs this many times the share of HBM
+// time that one element of a 128-row G tile costs its CTA (measured: an r x 64 tile takes about r * 64 * 0.18 ns of
+// one SM's ALUs, the 16 KB of a G tile 0.37 us of its share of HBM, and the ratio of the two per rank is about 0.045 / T).
+constexpr double K1_GENERATION_PER_RANK = 0.045;
+// Cost model of the decompression planner (microseconds on one SM): bytes an SM takes in per microsecond whatever their
+// source (about 60 GB/s with the tiles it can keep in flight), values of A per microsecond that the generator warps
+// make next to the streaming warps (8 or fewer warps), the share of a slab's generation that stays exposed with one
+// slab buffer (the combine warps help) or overlaps badly with two, and the fixed cost of an item.
+constexpr double K2_SM_BYTES_PER_US = 60e3;
+constexpr double K2_VALUES_PER_US_8_WARPS = 2000.0, K2_VALUES_PER_US_FEWER = 1300.0;
+constexpr double K2_EXPOSED_ONE_SLAB = 0.55, K2_OVERLAP_PENALTY = 0.35, K2_ITEM_OVERHEAD_US = 0.2;
 // Values of A that the generator warps of one SM produce while the SM streams one 64-column step of two G tiles
 // (about 0.6 us): the cluster is made large enough that a CTA's share of a tile stays below this.
 constexpr int PAIR_VALUES_PER_STEP = 2048;
@@ -408,7 +419,7 @@ inline void plan_compress(TcSet& set, const std::vector<flora_mat>& G, int r)
     uint32_t cols = 32;
     while ((int)cols < T * r_pad) cols <<= 1;
     // cluster size from the generation / load ratio
-    const double ratio = r * 0.045 / T;
+    const double ratio = r * K1_GENERATION_PER_RANK / T;
     int S = 1;
     while (S < 8 && ratio / S > 0.5) S <<= 1;
     while (S > 1 && (int64_t)S * T > 2 * max_tiles) S >>= 1;         // not more CTAs than there are rows to share
@@ -601,8 +612,8 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
     // r*bn normals at the generator warps' rate and overlaps the previous item's streaming
     // (an SM takes in about 60 GB/s whatever the source: the chunks of S count like the W tile itself)
     const double t_tile = std::max((double)bn * 128 * 4 / (6.5e6 / sm_count()),
-                                   ((double)bn * 128 * 2 + (double)kchunks * S_CHUNK_BYTES) / 60e3);
-    const double t_slab = (double)r * bn / (GW >= 8 ? 2000.0 : 1300.0);   // generator warps share the SM with the streaming warps
+                                   ((double)bn * 128 * 2 + (double)kchunks * S_CHUNK_BYTES) / K2_SM_BYTES_PER_US);
+    const double t_slab = (double)r * bn / (GW >= 8 ? K2_VALUES_PER_US_8_WARPS : K2_VALUES_PER_US_FEWER);   // generator warps share the SM with the streaming warps
     auto build = [&](int run, std::vector<K2Item>& out) {
         out.clear();
         for (size_t i = 0; i < W.size(); ++i) {
@@ -633,7 +644,8 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
         for (size_t k = 0; k < sorted.size(); ++k) {
             // generation overlaps the streaming of the previous item, but the two compete for issue slots
             const double stream = sorted[k].tiles * t_tile;
-            t[k % t.size()] += nslabs == 1 ? 0.55 * t_slab + stream + 0.2 : std::max(t_slab, stream) + 0.35 * std::min(t_slab, stream) + 0.2;
+            t[k % t.size()] += nslabs == 1 ? K2_EXPOSED_ONE_SLAB * t_slab + stream + K2_ITEM_OVERHEAD_US
+                                           : std::max(t_slab, stream) + K2_OVERLAP_PENALTY * std::min(t_slab, stream) + K2_ITEM_OVERHEAD_US;
         }
         return *std::max_element(t.begin(), t.end());
     };
