@@ -25,11 +25,12 @@
 namespace flora {
 
 constexpr int PAIR_T = 2;                   // 128-row tiles per CTA (accumulators: PAIR_T x N <= 512 tensor-memory columns)
-constexpr int PAIR_FIXED_WARPS = 4;         // warp 0: G loads, 1: MMA issue, 2: slice forwarding, 3: relay of the follower's barriers
+constexpr int PAIR_FIXED_WARPS = 4;         // single-thread roles on warps 0, 4, 8, 12: G loads; MMA issue (tile 0); slice forwarding;
+                                            // MMA issue (tile 1) in the leader, relay of the step's readiness in the follower
 constexpr int PAIR_EPI_WARPS = 8;           // two groups of four: group t writes out tile t; between two units they generate too
 constexpr int PAIR_MAX_GEN_WARPS = 16;
 constexpr int PAIR_MAX_THREADS = 32 * (PAIR_FIXED_WARPS + PAIR_MAX_GEN_WARPS + PAIR_EPI_WARPS);
-constexpr int PAIR_RELAY_DEPTH = 8;         // ring of the follower -> leader "stage ready" barriers (deeper than either tile ring)
+constexpr int PAIR_RELAY_DEPTH = 8;         // ring of the leader's per-step "operands ready" barriers (deeper than either tile ring)
 inline int pair_threads(int gen_warps) { return 32 * (PAIR_FIXED_WARPS + gen_warps + PAIR_EPI_WARPS); }
 
 struct PairSmem {
@@ -40,6 +41,8 @@ struct PairSmem {
     int next_item;      // generation work items handed out so far (one item = 32 tasks of one step's slice)
     int total_steps;    // 64-column steps of all units of this cluster
 };
+// full_g / full_a: in the follower, its G tiles / its half of an A tile have landed (its relay watches them); in the
+// leader the same arrivals and bytes go to ready[step % PAIR_RELAY_DEPTH], which the follower's relay completes.
 
 // N: columns of the accumulators = r rounded up to a multiple of 64 (rows r .. N of A are zero).
 // A CTA of rank q in its cluster belongs to pair q / 2 and holds half h = q % 2 of every A tile: rows
