@@ -15,6 +15,7 @@
 #include <new>
 
 #include "flora_pair.cuh"
+#include "flora_pair_k2.cuh"
 #include "flora_pool.cuh"
 #include "flora_tc.cuh"
 
@@ -47,6 +48,7 @@ struct TcSet {
     // decompression
     int bn = 128, slots = 2, cstages = 2, k2_gw = 8, k2_nslabs = 2, k2_grid_max = 148;
     bool k2_bf16 = false;               // ranks above 64: the kernel reads a bf16 copy of the sketches
+    bool k2_pair = false;               // ... and runs on CTA pairs (decompress_pair_kernel); k2_grid_max then counts pairs
     __nv_bfloat16* d_sb = nullptr;      // that copy (scratch owned by the set)
     std::vector<int> k2_launch_first_mat;
     size_t k2_smem = 0;
@@ -607,7 +609,29 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
     set.k2_gw = GW;
     set.k2_nslabs = nslabs;
     set.k2_smem = nslabs * slab_bytes + (size_t)cstages * S_CHUNK_BYTES + (size_t)slots * slot + sizeof(K2Smem) + 1024;
-    const int grid_max = sm_count() * per_sm;
+    int grid_max = sm_count() * per_sm;
+    // Ranks whose slab leaves one CTA room for a single buffer run on CTA pairs: each CTA holds half of a 128-column slab (two buffers of kchunks x 8 KB), the
+    // sketch chunks of its own tiles (as many stages as fit beside two W tiles, at most two tiles' worth) and its W tiles.
+    // (where one CTA has room for two slab buffers itself, up to r = 192, it is the faster of the two: measured)
+    const bool pair = bf16s && tune_knob("FLORA_K2_PAIR", nslabs == 1 ? 1 : 0, 0, 1) != 0;
+    set.k2_pair = pair;
+    if (pair) {
+        const size_t half_slab = (size_t)kchunks * 64 * 128, pslot = 2 * (size_t)W_BOX_BYTES;
+        const size_t pbudget = SMEM_BUDGET - sizeof(K2PairSmem) - 1024 - 2 * half_slab;
+        int pc = std::min(K2_MAX_CSTAGES, 2 * kchunks);
+        pc = tune_knob("FLORA_K2_CSTAGES", pc, 2, K2_MAX_CSTAGES);
+        while (pc > 2 && (size_t)pc * S_CHUNK_BYTES + 2 * pslot > pbudget) --pc;
+        int ps = (int)std::min<size_t>(K2_MAX_SLOTS, (pbudget - (size_t)pc * S_CHUNK_BYTES) / pslot);
+        ps = tune_knob("FLORA_K2_SLOTS", ps, 2, std::max(2, ps));
+        bn = set.bn = K2P_BN;
+        nslabs = set.k2_nslabs = 2;
+        cstages = set.cstages = pc;
+        slots = set.slots = ps;
+        GW = set.k2_gw = K2P_GEN_WARPS;
+        set.k2_smem = decompress_pair_smem_bytes(r, ps, pc);
+        grid_max = std::max(1, sm_count() / 2);
+    }
+    const double pair_f = pair ? 0.5 : 1.0;          // a pair streams an item's tiles two at a time, and each CTA generates half a slab
     // cost model (microseconds of one SM): a tile streams bn*128*4 bytes at the SM's share of HBM; a slab costs
     // r*bn normals at the generator warps' rate and overlaps the previous item's streaming
     // (an SM takes in about 60 GB/s whatever the source: the chunks of S count like the W tile itself)
@@ -643,9 +667,9 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
         std::vector<double> t((size_t)std::max(grid, 1), 0.0);
         for (size_t k = 0; k < sorted.size(); ++k) {
             // generation overlaps the streaming of the previous item, but the two compete for issue slots
-            const double stream = sorted[k].tiles * t_tile;
-            t[k % t.size()] += nslabs == 1 ? K2_EXPOSED_ONE_SLAB * t_slab + stream + K2_ITEM_OVERHEAD_US
-                                           : std::max(t_slab, stream) + K2_OVERLAP_PENALTY * std::min(t_slab, stream) + K2_ITEM_OVERHEAD_US;
+            const double stream = (pair ? (sorted[k].tiles + 1) / 2 : sorted[k].tiles) * t_tile, gen = pair_f * t_slab;
+            t[k % t.size()] += nslabs == 1 ? K2_EXPOSED_ONE_SLAB * gen + stream + K2_ITEM_OVERHEAD_US
+                                           : std::max(gen, stream) + K2_OVERLAP_PENALTY * std::min(gen, stream) + K2_ITEM_OVERHEAD_US;
         }
         return *std::max_element(t.begin(), t.end());
     };
@@ -998,7 +1022,9 @@ inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float s
             launches.fetch_add(1, std::memory_order_relaxed);
         }
     }
-    if (!(set.k2_bf16 ? raise_smem_limit<decompress_tc_kernel<true>>() : raise_smem_limit<decompress_tc_kernel<false>>())) return FLORA_ERR_CUDA;
+    if (!(set.k2_pair ? raise_smem_limit<decompress_pair_kernel>()
+                      : set.k2_bf16 ? raise_smem_limit<decompress_tc_kernel<true>>() : raise_smem_limit<decompress_tc_kernel<false>>()))
+        return FLORA_ERR_CUDA;
     for (size_t l = 0; l + 1 < set.k2_launch_begin.size(); ++l) {
         const int begin = set.k2_launch_begin[l], end = set.k2_launch_begin[l + 1];
         if (end == begin) continue;
@@ -1006,7 +1032,25 @@ inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float s
         SeedTable table;
         for (int i = 0; i < SEEDS_PER_LAUNCH; ++i) table.s[i] = seed_base + i < set.count ? seeds[seed_base + i] : 0;
         const int grid = std::min(set.k2_grid_max, end - begin);
-        if (set.k2_bf16)
+        if (set.k2_pair) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)(2 * grid));                // `grid` pairs
+            cfg.blockDim = dim3((unsigned)K2P_THREADS);
+            cfg.dynamicSmemBytes = set.k2_smem;
+            cfg.stream = st;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 2;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            const TcMatrix* mats = set.d_mats;
+            const K2Item* items = set.d_k2 + begin;
+            if (cudaLaunchKernelEx(&cfg, decompress_pair_kernel, mats, items, end - begin, table, seed_base, r, scale, step, set.slots, set.cstages) !=
+                cudaSuccess)
+                return FLORA_ERR_CUDA;
+        } else if (set.k2_bf16)
             decompress_tc_kernel<true><<<grid, 32 * (K2_FIXED_WARPS + set.k2_gw), set.k2_smem, st>>>(
                 set.d_mats, set.d_k2 + begin, end - begin, table, seed_base, r, scale, step, set.bn, set.slots, set.cstages, set.k2_gw, set.k2_nslabs);
         else
