@@ -29,7 +29,7 @@ constexpr int K2P_BN = 128;           // columns of a slab (64 per CTA)
 
 struct K2PairSmem {
     uint64_t w_full[K2_MAX_SLOTS], w_free[K2_MAX_SLOTS], out_ready[K2_MAX_SLOTS];
-    uint64_t c_full[K2_MAX_CSTAGES], c_empty[K2_MAX_CSTAGES], peer_c[K2_MAX_CSTAGES], acc_full[2], acc_empty[2], slab_full[2], slab_empty[2];
+    uint64_t c_full[K2_MAX_CSTAGES], c_empty[K2_MAX_CSTAGES], acc_full[2], acc_empty[2], slab_full[2], slab_empty[2];
     uint32_t tmem_base;
     int abort;
 };
@@ -62,9 +62,9 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
             ptx::mbar_init(ptx::smem_addr(&ctl->out_ready[s]), 8);
         }
         for (int s = 0; s < cstages; ++s) {
-            ptx::mbar_init(ptx::smem_addr(&ctl->c_full[s]), 1);
+            // the leader's barrier of a stage also takes the follower's word that its own chunk has landed: one wait per chunk
+            ptx::mbar_init(ptx::smem_addr(&ctl->c_full[s]), half == 0 ? 2 : 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->c_empty[s]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctl->peer_c[s]), 1);
         }
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->acc_full[s]), 1);
@@ -162,8 +162,7 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
                     ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[gt & 1]), (((uint32_t)gt >> 1) & 1u) ^ 1u, abort);
                     for (int kc = 0; kc < kchunks && ok; ++kc, pc.advance(cstages)) {
                         const int s = pc.s;
-                        ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[s]), pc.wraps & 1u, abort) &&
-                             ptx::mbar_wait(ptx::smem_addr(&ctl->peer_c[s]), pc.wraps & 1u, abort);
+                        ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[s]), pc.wraps & 1u, abort);
                         if (!ok) break;
                         ptx::tc_fence_after_sync();
 #pragma unroll
@@ -189,7 +188,7 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
                 for (int c = 0; c < iterations(item) * kchunks; ++c, pc.advance(cstages)) {
                     ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[pc.s]), pc.wraps & 1u, abort);
                     if (!ok) break;
-                    ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_addr(&ctl->peer_c[pc.s]), 0u));
+                    ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_addr(&ctl->c_full[pc.s]), 0u));
                 }
             }
         }
