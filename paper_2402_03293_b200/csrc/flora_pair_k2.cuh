@@ -7,8 +7,11 @@
 // buffers fit and the slab of the next item is generated while the current item streams, which a single CTA
 // cannot do above r = 192.  The pair takes the row tiles of an item in turn (the leader the even ones), so an item
 // streams in half the time and each CTA generates half as much per item.  Each CTA loads, combines and stores its
-// own W tiles; the leader's one thread issues the MMAs for both and learns from a relay thread of the follower
-// that the follower's sketch chunks have landed.
+// own W tiles.  The leader issues the MMAs for both, from two threads: a thread gets an MMA accepted only about every
+// hundred cycles, and with sixteen of them and five commits per tile iteration one thread alone sets the pace of the
+// kernel.  The two take the tile iterations in turn, each with two of the four accumulators and its own ring of sketch
+// chunks, filled in step with the other's, and each learns from a relay thread of the follower that the follower's
+// chunks have landed.
 // The sketch is read from its bf16 copy (see sketch_to_bf16_kernel).  All waits are bounded.
 #pragma once
 #include <cuda.h>
@@ -22,20 +25,29 @@
 
 namespace flora {
 
-constexpr int K2P_FIXED_WARPS = 12;   // warp 0: W loads, 1: MMA issue (leader) / relay (follower), 2-5 and 8-11: combine, 6: S loads, 7: W stores
+constexpr int K2P_FIXED_WARPS = 12;   // warp 0: W loads and stores, 1 and 7: MMA issue (leader) / relay (follower), 2-5 and 8-11: combine, 6: S loads
 constexpr int K2P_GEN_WARPS = 8;      // warps 12..19: slab generators
 constexpr int K2P_THREADS = 32 * (K2P_FIXED_WARPS + K2P_GEN_WARPS);
 constexpr int K2P_BN = 128;           // columns of a slab (64 per CTA)
+constexpr int K2P_ACCS = 4;           // accumulators in tensor memory: two per MMA-issuing thread
 
 struct K2PairSmem {
-    uint64_t w_full[K2_MAX_SLOTS], w_free[K2_MAX_SLOTS], out_ready[K2_MAX_SLOTS];
-    uint64_t c_full[K2_MAX_CSTAGES], c_empty[K2_MAX_CSTAGES], acc_full[2], acc_empty[2], slab_full[2], slab_empty[2];
+    uint64_t w_full[K2_MAX_SLOTS], out_ready[K2_MAX_SLOTS];
+    uint64_t c_full[K2_MAX_CSTAGES], c_empty[K2_MAX_CSTAGES], acc_full[K2P_ACCS], acc_empty[K2P_ACCS], slab_full[2], slab_empty[2];
     uint32_t tmem_base;
     int abort;
 };
 
+// A role's position in its cluster's sequence of tile iterations: item `it` (the k-th of this cluster), iteration p of n.
+struct K2Cursor {
+    int it, k, p, n;
+    K2Item item;
+};
+
 // Cluster c (two CTAs) processes the items c, c + clusters, ...; within an item, tile iteration p covers the row tiles
 // 2p (leader) and 2p + 1 (follower; it may not exist, then the follower loads and stores nothing for that iteration).
+// Iterations are numbered through all items of the cluster (gt); the even ones belong to the first MMA thread, its
+// ring of sketch chunks (cstages / 2 stages) and accumulators 0 and 2, the odd ones to the second.
 __global__ void __launch_bounds__(K2P_THREADS, 1)
 decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict__ items, int n_items, const __grid_constant__ SeedTable seeds,
                        int seed_base, int r, float scale, float step, int slots, int cstages)
@@ -53,12 +65,12 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t half = ptx::cluster_ctarank();
     const int cluster = (int)(blockIdx.x >> 1), clusters = (int)(gridDim.x >> 1);
-    const uint32_t tmem_cols = 2u * K2P_BN;
+    const uint32_t tmem_cols = (uint32_t)K2P_ACCS * K2P_BN;
+    const int ring_stages = cstages >> 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < slots; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->w_full[s]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctl->w_free[s]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->out_ready[s]), 8);
         }
         for (int s = 0; s < cstages; ++s) {
@@ -66,11 +78,13 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
             ptx::mbar_init(ptx::smem_addr(&ctl->c_full[s]), half == 0 ? 2 : 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->c_empty[s]), 1);
         }
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < K2P_ACCS; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->acc_full[s]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[s]), 16);                 // the eight combine warps of both CTAs (leader's barrier)
+        }
+        for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->slab_full[s]), 2 * K2P_GEN_WARPS);  // the generator warps of both CTAs (leader's barrier)
-            ptx::mbar_init(ptx::smem_addr(&ctl->slab_empty[s]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctl->slab_empty[s]), 2);                 // both MMA threads are done with the slab
         }
         ctl->abort = 0;
         ptx::fence_barrier_init();
@@ -89,80 +103,152 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
     // tile iterations of an item, and whether this CTA has a tile in iteration p
     auto iterations = [](const K2Item& it) { return (it.tiles + 1) >> 1; };
     auto has_tile = [&](const K2Item& it, int p) { return 2 * p + (int)half < it.tiles; };
+    auto cur_load = [&](K2Cursor& c) {
+        if (c.it < n_items) {
+            c.item = items[c.it];
+            c.n = iterations(c.item);
+        }
+    };
+    // carries an iteration index that ran past the end of its item into the items that follow
+    auto cur_norm = [&](K2Cursor& c) {
+        while (c.it < n_items && c.p >= c.n) {
+            c.p -= c.n;
+            c.it += clusters;
+            ++c.k;
+            cur_load(c);
+        }
+    };
+    auto cur_init = [&](K2Cursor& c, int first) {
+        c.it = cluster;
+        c.k = 0;
+        c.p = first;
+        c.n = 0;
+        cur_load(c);
+        cur_norm(c);
+    };
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ W tile loads
+        // ------------------------------------------------------------------ W tile loads and stores
+        // One thread: the tile of iteration gt + slots goes into the slot of iteration gt as soon as the store of that one
+        // has read it out, which this thread is the one to know.
         if (lane == 0) {
-            RingPos pw;
+            K2Cursor ld, stc;
+            cur_init(ld, 0);
+            cur_init(stc, 0);
+            RingPos pl, ps;
             int issued = 0;
-            bool ok = true;
-            for (int it = cluster; it < n_items && ok; it += clusters) {
-                const K2Item item = items[it];
-                const TcMatrix* mat = mats + item.mat;
-                const int live_boxes = min(2, (mat->m - item.col0 + 63) >> 6);
-                for (int p = 0; p < iterations(item); ++p, pw.advance(slots), ++issued) {
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->w_free[pw.s]), (pw.wraps & 1u) ^ 1u, abort);
-                    if (!ok) break;
-                    const uint32_t bar = ptx::smem_addr(&ctl->w_full[pw.s]);
-                    if (has_tile(item, p)) {
-                        ptx::mbar_arrive_expect_tx(bar, (uint32_t)live_boxes * W_BOX_BYTES);
-                        for (int bx = 0; bx < live_boxes; ++bx)
-                            ptx::tma_load_2d(w_ring + pw.s * slot_bytes + bx * W_BOX_BYTES, &mat->map_w, item.col0 + bx * 64, item.row0 + (2 * p + (int)half) * 128, bar);
-                    } else {
-                        ptx::mbar_arrive(bar);
-                    }
+            auto issue_load = [&]() {
+                const TcMatrix* mat = mats + ld.item.mat;
+                const int live_boxes = min(2, (mat->m - ld.item.col0 + 63) >> 6);
+                const uint32_t bar = ptx::smem_addr(&ctl->w_full[pl.s]);
+                if (has_tile(ld.item, ld.p)) {
+                    ptx::mbar_arrive_expect_tx(bar, (uint32_t)live_boxes * W_BOX_BYTES);
+                    for (int bx = 0; bx < live_boxes; ++bx)
+                        ptx::tma_load_2d(w_ring + pl.s * slot_bytes + bx * W_BOX_BYTES, &mat->map_w, ld.item.col0 + bx * 64,
+                                         ld.item.row0 + (2 * ld.p + (int)half) * 128, bar);
+                } else {
+                    ptx::mbar_arrive(bar);
                 }
+                ++ld.p;
+                cur_norm(ld);
+                pl.advance(slots);
+                ++issued;
+            };
+            for (int i = 0; i < slots && ld.it < n_items; ++i) issue_load();
+            bool ok = true;
+            while (stc.it < n_items) {
+                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->out_ready[ps.s]), ps.wraps & 1u, abort);
+                if (!ok) break;
+                if (has_tile(stc.item, stc.p)) {
+                    const TcMatrix* mat = mats + stc.item.mat;
+                    const int live_boxes = min(2, (mat->m - stc.item.col0 + 63) >> 6);
+                    for (int bx = 0; bx < live_boxes; ++bx)
+                        ptx::tma_store_2d(&mat->map_w, stc.item.col0 + bx * 64, stc.item.row0 + (2 * stc.p + (int)half) * 128,
+                                          w_ring + ps.s * slot_bytes + bx * W_BOX_BYTES);
+                    ptx::tma_store_commit();
+                    ptx::tma_store_wait_read<0>();          // the slot has been read out: it can be refilled
+                }
+                ++stc.p;
+                cur_norm(stc);
+                ps.advance(slots);
+                if (ld.it < n_items) issue_load();
             }
+            ptx::tma_store_wait_all<0>();
             if (*abort)   // loads that nobody consumed: wait (bounded) until they have landed
                 for (int g = max(0, issued - slots); g < issued; ++g) ptx::mbar_wait(ptx::smem_addr(&ctl->w_full[g % slots]), (uint32_t)(g / slots) & 1u, abort);
         }
     } else if (warp == 6) {
         // ------------------------------------------------------------------ S chunk loads (bf16 copy, 64 values of the rank each)
         if (lane == 0) {
-            RingPos pc;
+            // the chunks of an even and of the following odd iteration in turn, each into its thread's ring, so that both
+            // MMA threads always have chunks to work on
+            K2Cursor cs[2];
+            cur_init(cs[0], 0);
+            cur_init(cs[1], 1);
+            RingPos prs[2];
             bool ok = true;
-            for (int it = cluster; it < n_items && ok; it += clusters) {
-                const K2Item item = items[it];
-                const TcMatrix* mat = mats + item.mat;
-                for (int p = 0; p < iterations(item) && ok; ++p) {
-                    for (int kc = 0; kc < kchunks; ++kc, pc.advance(cstages)) {
-                        ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_empty[pc.s]), (pc.wraps & 1u) ^ 1u, abort);
+            while (ok && (cs[0].it < n_items || cs[1].it < n_items)) {
+                for (int kc = 0; kc < kchunks && ok; ++kc) {
+#pragma unroll
+                    for (int x = 0; x < 2; ++x) {
+                        if (cs[x].it >= n_items) continue;
+                        const int st = x * ring_stages + prs[x].s;
+                        ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_empty[st]), (prs[x].wraps & 1u) ^ 1u, abort);
                         if (!ok) break;
-                        const uint32_t bar = ptx::smem_addr(&ctl->c_full[pc.s]);
-                        if (has_tile(item, p)) {
+                        const uint32_t bar = ptx::smem_addr(&ctl->c_full[st]);
+                        if (has_tile(cs[x].item, cs[x].p)) {
                             ptx::mbar_arrive_expect_tx(bar, S_CHUNK_BYTES);
-                            ptx::tma_load_2d(c_ring + pc.s * S_CHUNK_BYTES, &mat->map_sb, kc * 64, item.row0 + (2 * p + (int)half) * 128, bar);
+                            ptx::tma_load_2d(c_ring + st * S_CHUNK_BYTES, &mats[cs[x].item.mat].map_sb, kc * 64,
+                                             cs[x].item.row0 + (2 * cs[x].p + (int)half) * 128, bar);
                         } else {
                             ptx::mbar_arrive(bar);
                         }
+                        prs[x].advance(ring_stages);
                     }
+                }
+#pragma unroll
+                for (int x = 0; x < 2; ++x) {
+                    cs[x].p += 2;
+                    cur_norm(cs[x]);
                 }
             }
             if (*abort)
-                for (int s = 0; s < cstages; ++s) {
-                    const uint32_t fills = pc.wraps + (s < pc.s ? 1u : 0u);
-                    if (fills) ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[s]), (fills - 1u) & 1u, abort);
-                }
+                for (int x = 0; x < 2; ++x)
+                    for (int s = 0; s < ring_stages; ++s) {
+                        const uint32_t fills = prs[x].wraps + (s < prs[x].s ? 1u : 0u);
+                        if (fills) ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[x * ring_stages + s]), (fills - 1u) & 1u, abort);
+                    }
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || warp == 7) {
+        const int x = warp == 1 ? 0 : 1;                    // which of the two issuing threads (leader) or relays (follower)
         if (lane == 0 && half == 0) {
-            // -------------------------------------------------------------- MMA issuer (the pair's leader)
+            // -------------------------------------------------------------- MMA issuers (the pair's leader)
+            // A thread waits for the slab of every item it passes, also of one in which the other thread has all the
+            // iterations, and commits to slab_empty when it leaves: every phase of those barriers is then seen by
+            // both, in order, which waiting by parity relies on.
             const uint32_t idesc = ptx::umma_idesc_bf16_mn(256u, (uint32_t)K2P_BN);
-            const uint64_t desc_ring = ptx::umma_desc_k_sw128(c_ring);
+            const uint64_t desc_ring = ptx::umma_desc_k_sw128(c_ring + (uint32_t)(x * ring_stages) * (uint32_t)S_CHUNK_BYTES);
+            K2Cursor c;
+            c.it = cluster;
+            c.k = 0;
+            c.p = x;
+            c.n = 0;
+            cur_load(c);
             RingPos pc;
-            int gt = 0, k = 0;
+            int gt = x;
             bool ok = true;
-            for (int it = cluster; it < n_items && ok; it += clusters, ++k) {
-                const K2Item item = items[it];
-                const int sb = k & 1;
+            while (ok && c.it < n_items) {
+                const int sb = c.k & 1;
                 const uint64_t desc_slab = ptx::umma_desc_k_sw128(slab0 + sb * slab_bytes);
-                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_full[sb]), (uint32_t)(k >> 1) & 1u, abort);     // both halves of the slab are written
-                for (int p = 0; p < iterations(item) && ok; ++p, ++gt) {
-                    const uint32_t acc_addr = tmem + (uint32_t)(gt & 1) * K2P_BN;
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[gt & 1]), (((uint32_t)gt >> 1) & 1u) ^ 1u, abort);
-                    for (int kc = 0; kc < kchunks && ok; ++kc, pc.advance(cstages)) {
+                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_full[sb]), (uint32_t)(c.k >> 1) & 1u, abort);     // both halves of the slab are written
+                for (; c.p < c.n && ok; c.p += 2, gt += 2) {
+                    const int a = gt & (K2P_ACCS - 1);
+                    const uint32_t acc_addr = tmem + (uint32_t)a * K2P_BN;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[a]), (((uint32_t)gt >> 2) & 1u) ^ 1u, abort);
+                    for (int kc = 0; kc < kchunks && ok; ++kc, pc.advance(ring_stages)) {
                         const int s = pc.s;
-                        ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[s]), pc.wraps & 1u, abort);
+                        const uint32_t full = ptx::smem_addr(&ctl->c_full[x * ring_stages + s]);
+                        ok = ptx::mbar_wait(full, pc.wraps & 1u, abort);
                         if (!ok) break;
                         ptx::tc_fence_after_sync();
 #pragma unroll
@@ -173,47 +259,32 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
                             const uint64_t db = desc_slab + (uint64_t)((kc * slab_block + k16 * 32) >> 4);
                             ptx::umma_bf16_pair(acc_addr, da, db, idesc, (kc | k16) != 0);
                         }
-                        ptx::umma_commit_pair(ptx::smem_addr(&ctl->c_empty[s]), (uint16_t)3u);
+                        ptx::umma_commit_pair(ptx::smem_addr(&ctl->c_empty[x * ring_stages + s]), (uint16_t)3u);
                     }
-                    if (ok) ptx::umma_commit_pair(ptx::smem_addr(&ctl->acc_full[gt & 1]), (uint16_t)3u);
+                    if (ok) ptx::umma_commit_pair(ptx::smem_addr(&ctl->acc_full[a]), (uint16_t)3u);
                 }
-                if (ok) ptx::umma_commit_pair(ptx::smem_addr(&ctl->slab_empty[sb]), (uint16_t)3u);   // every MMA that reads this slab has completed
+                if (ok) ptx::umma_commit_pair(ptx::smem_addr(&ctl->slab_empty[sb]), (uint16_t)3u);   // every MMA of this thread that reads the slab has completed
+                c.p -= c.n;
+                c.it += clusters;
+                ++c.k;
+                cur_load(c);
             }
         } else if (lane == 0) {
-            // -------------------------------------------------------------- relay (the follower): its sketch chunk has landed
+            // -------------------------------------------------------------- relays (the follower): a sketch chunk has landed
+            K2Cursor c;
+            cur_init(c, x);
             RingPos pc;
             bool ok = true;
-            for (int it = cluster; it < n_items && ok; it += clusters) {
-                const K2Item item = items[it];
-                for (int c = 0; c < iterations(item) * kchunks; ++c, pc.advance(cstages)) {
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->c_full[pc.s]), pc.wraps & 1u, abort);
+            while (ok && c.it < n_items) {
+                for (int kc = 0; kc < kchunks; ++kc, pc.advance(ring_stages)) {
+                    const uint32_t bar = ptx::smem_addr(&ctl->c_full[x * ring_stages + pc.s]);
+                    ok = ptx::mbar_wait(bar, pc.wraps & 1u, abort);
                     if (!ok) break;
-                    ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_addr(&ctl->c_full[pc.s]), 0u));
+                    ptx::mbar_arrive_cluster(ptx::map_to_cta(bar, 0u));
                 }
+                c.p += 2;
+                cur_norm(c);
             }
-        }
-    } else if (warp == 7) {
-        // ------------------------------------------------------------------ W tile stores
-        if (lane == 0) {
-            RingPos pw;
-            bool ok = true;
-            for (int it = cluster; it < n_items && ok; it += clusters) {
-                const K2Item item = items[it];
-                const TcMatrix* mat = mats + item.mat;
-                const int live_boxes = min(2, (mat->m - item.col0 + 63) >> 6);
-                for (int p = 0; p < iterations(item); ++p, pw.advance(slots)) {
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->out_ready[pw.s]), pw.wraps & 1u, abort);
-                    if (!ok) break;
-                    if (has_tile(item, p)) {
-                        for (int bx = 0; bx < live_boxes; ++bx)
-                            ptx::tma_store_2d(&mat->map_w, item.col0 + bx * 64, item.row0 + (2 * p + (int)half) * 128, w_ring + pw.s * slot_bytes + bx * W_BOX_BYTES);
-                        ptx::tma_store_commit();
-                        ptx::tma_store_wait_read<0>();          // the slot has been read out: it can be refilled
-                    }
-                    ptx::mbar_arrive(ptx::smem_addr(&ctl->w_free[pw.s]));
-                }
-            }
-            ptx::tma_store_wait_all<0>();
         }
     } else if ((warp >= 2 && warp <= 5) || (warp >= 8 && warp <= 11)) {
         // ------------------------------------------------------------------ combine the accumulator with the W tile
@@ -233,7 +304,8 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
             const int mine = max(0, min(4, live_chunks - c_begin));
             for (int p = 0; p < iterations(item); ++p, ++gt, pw.advance(slots)) {
                 const int s = pw.s;
-                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[gt & 1]), ((uint32_t)gt >> 1) & 1u, abort) &&
+                const int a = gt & (K2P_ACCS - 1);
+                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[a]), ((uint32_t)gt >> 2) & 1u, abort) &&
                      ptx::mbar_wait(ptx::smem_addr(&ctl->w_full[s]), pw.wraps & 1u, abort);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
@@ -242,7 +314,7 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
                     uint32_t acc[4][16];
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
-                        if (k < mine) ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(gt & 1) * K2P_BN + (c_begin + k) * 16, acc[k]);
+                        if (k < mine) ptx::tmem_ld_16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)a * K2P_BN + (c_begin + k) * 16, acc[k]);
                     ptx::tmem_ld_wait();
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
@@ -271,7 +343,7 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    const uint32_t ebar = ptx::smem_addr(&ctl->acc_empty[gt & 1]);
+                    const uint32_t ebar = ptx::smem_addr(&ctl->acc_empty[a]);
                     if (half == 0) ptx::mbar_arrive(ebar);
                     else ptx::mbar_arrive_cluster(ptx::map_to_cta(ebar, 0u));
                     ptx::mbar_arrive(ptx::smem_addr(&ctl->out_ready[s]));

@@ -621,6 +621,7 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
         int pc = std::min(K2_MAX_CSTAGES, 2 * kchunks);
         pc = tune_knob("FLORA_K2_CSTAGES", pc, 2, K2_MAX_CSTAGES);
         while (pc > 2 && (size_t)pc * S_CHUNK_BYTES + 2 * pslot > pbudget) --pc;
+        pc &= ~1;                                        // two rings of equal depth, one per MMA-issuing thread
         int ps = (int)std::min<size_t>(K2_MAX_SLOTS, (pbudget - (size_t)pc * S_CHUNK_BYTES) / pslot);
         ps = tune_knob("FLORA_K2_SLOTS", ps, 2, std::max(2, ps));
         bn = set.bn = K2P_BN;
