@@ -29,6 +29,7 @@ constexpr int K2P_FIXED_WARPS = 12;   // warp 0: W loads and stores, 1 and 7: MM
 constexpr int K2P_GEN_WARPS = 8;      // warps 12..19: slab generators
 constexpr int K2P_THREADS = 32 * (K2P_FIXED_WARPS + K2P_GEN_WARPS);
 constexpr int K2P_BN = 128;           // columns of a slab (64 per CTA)
+constexpr int K2P_PREFETCH_AHEAD = 2; // W tiles asked into L2 this many tile iterations before their slot comes free
 constexpr int K2P_ACCS = 4;           // accumulators in tensor memory: two per MMA-issuing thread
 
 struct K2PairSmem {
@@ -132,9 +133,10 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
         // One thread: the tile of iteration gt + slots goes into the slot of iteration gt as soon as the store of that one
         // has read it out, which this thread is the one to know.
         if (lane == 0) {
-            K2Cursor ld, stc;
+            K2Cursor ld, stc, pf;
             cur_init(ld, 0);
             cur_init(stc, 0);
+            cur_init(pf, slots + K2P_PREFETCH_AHEAD);       // this far ahead of the loads, tiles are asked into L2
             RingPos pl, ps;
             int issued = 0;
             auto issue_load = [&]() {
@@ -153,6 +155,16 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
                 cur_norm(ld);
                 pl.advance(slots);
                 ++issued;
+                if (pf.it < n_items) {
+                    if (has_tile(pf.item, pf.p)) {
+                        const TcMatrix* pmat = mats + pf.item.mat;
+                        const int pboxes = min(2, (pmat->m - pf.item.col0 + 63) >> 6);
+                        for (int bx = 0; bx < pboxes; ++bx)
+                            ptx::tma_prefetch_l2_2d(&pmat->map_w, pf.item.col0 + bx * 64, pf.item.row0 + (2 * pf.p + (int)half) * 128);
+                    }
+                    ++pf.p;
+                    cur_norm(pf);
+                }
             };
             for (int i = 0; i < slots && ld.it < n_items; ++i) issue_load();
             bool ok = true;

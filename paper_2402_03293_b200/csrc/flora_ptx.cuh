@@ -138,6 +138,12 @@ __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepco
 // Lets the next kernel of the stream begin its own set-up as soon as resources free up.
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Asks for a tile to be brought into L2 (no shared memory, no barrier): a later tma_load_2d of it finds it there.
+__device__ __forceinline__ void tma_prefetch_l2_2d(const void* tmap, int x, int y)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tmap), "r"(x), "r"(y) : "memory");
+}
+
 // ---------------------------------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem()
 {
