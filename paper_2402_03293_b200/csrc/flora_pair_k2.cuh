@@ -29,7 +29,7 @@ constexpr int K2P_FIXED_WARPS = 12;   // warp 0: W loads and stores, 1 and 7: MM
 constexpr int K2P_GEN_WARPS = 8;      // warps 12..19: slab generators
 constexpr int K2P_THREADS = 32 * (K2P_FIXED_WARPS + K2P_GEN_WARPS);
 constexpr int K2P_BN = 128;           // columns of a slab (64 per CTA)
-constexpr int K2P_PREFETCH_AHEAD = 2; // W tiles asked into L2 this many tile iterations before their slot comes free
+constexpr int K2P_PREFETCH_AHEAD = 0; // a W tile is asked into L2 when the tile before it in its slot is loaded (asking earlier was slower: measured)
 constexpr int K2P_ACCS = 4;           // accumulators in tensor memory: two per MMA-issuing thread
 
 struct K2PairSmem {
@@ -136,7 +136,7 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
             K2Cursor ld, stc, pf;
             cur_init(ld, 0);
             cur_init(stc, 0);
-            cur_init(pf, slots + K2P_PREFETCH_AHEAD);       // this far ahead of the loads, tiles are asked into L2
+            cur_init(pf, slots + K2P_PREFETCH_AHEAD);       // this far ahead of the loads, tiles are asked into L2: the slot's wait is then not for HBM
             RingPos pl, ps;
             int issued = 0;
             auto issue_load = [&]() {
