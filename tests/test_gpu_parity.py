@@ -236,6 +236,30 @@ def test_set_on_tensor_core_eligible_shapes():
     fset.close()
 
 
+@pytest.mark.parametrize("r", [200, 256])
+def test_set_decompress_on_cta_pairs_many_short_items(r):
+    """Ranks above 192 decompress on CTA pairs whose two MMA-issuing threads take tile iterations in turn across item
+    boundaries: a set with more column slabs than there are pairs, of matrices with 1 to 7 row tiles (odd and even
+    counts, ragged last tiles, a last slab of 8 to 72 live columns), compared element by element with the oracle."""
+    rng = np.random.default_rng(77)
+    shapes = [(int(rng.integers(1, 8)) * 128 - int(rng.integers(0, 120)), int(rng.integers(2, 7)) * 128 + int(rng.choice([8, 64, 72, 128])))
+              for _ in range(64)]
+    G, W, S = _small_set("bf16", r, shapes)
+    for i, s_ in enumerate(S):
+        s_.copy_(torch.from_numpy(np.random.default_rng(500 + i).standard_normal(tuple(s_.shape)).astype(np.float32)))
+    W0 = [w.clone() for w in W]
+    fset = fb.FloraSet(G, W, S)
+    seeds = [fb.flora_derive_seed(21, i, 0) for i in range(len(shapes))]
+    fset.decompress_apply(seeds, 0.02, 1.0)
+    torch.cuda.synchronize()
+    for i in range(len(shapes)):
+        ref = oracle_decompress(W0[i], S[i], seeds[i], 0.02, 1.0)
+        w0 = values(wl.as_numpy(W0[i])).astype(np.float64)
+        assert rel_err(values(wl.as_numpy(W[i])), values(ref)) <= TOL["bf16"], (i, shapes[i])
+        assert rel_err(values(wl.as_numpy(W[i])) - w0, values(ref) - w0) <= TOL["bf16"], (i, shapes[i])
+    fset.close()
+
+
 def test_host_to_device_entry_points():
     shapes = [(64, 160), (40, 72)]
     r = 8
