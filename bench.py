@@ -443,9 +443,11 @@ def run_flora(args):
         kinds[k] = 1e3 * total / shared_counts[k]                    # microseconds per launch group of that kind
     costs = op_costs(w, r)
     hbm, tf, src = measured_peaks()
-    names = {"compress": "compress kernel (C += G A^T), one launch over the weight set", "momentum": "compress kernel as the momentum update",
+    k1 = "compress_pair_kernel" if r > 64 else "compress_tc_kernel"
+    k2 = "decompress_pair_kernel" if r > 192 else "decompress_tc_kernel"
+    names = {"compress": k1 + " (C += G A^T), one launch over the weight set", "momentum": k1 + " as the momentum update",
              "momentum_resampled": "gram + apply + compress kernels (Algorithm 2's resampling step)",
-             "decompress": "decompress_tc_kernel (W -= lr S A), one launch over the weight set",
+             "decompress": ("sketch_to_bf16_kernel + " if r > 64 else "") + k2 + " (W -= lr S A), one launch over the weight set",
              "transfer": "gram + apply kernels (M <- M A_old A_new^T)", "transfer_axpby": "gram + apply kernels (M <- beta M + a C A_acc A_mom^T)"}
     main_kind = "compress" if "compress" in kinds else ("momentum" if "momentum" in kinds else "momentum_resampled")
     roofline = roofline_block(names[main_kind], costs[main_kind][0], costs[main_kind][1], kinds[main_kind], hbm, tf, src)
