@@ -56,6 +56,7 @@ def op_costs(w: wl.Workload, r: int):
     transfer_flops = sum(2 * r * r * m + 2 * n * r * r for n, m in w.shapes)
     return {
         "compress": (w.elements * eb + 2 * state, flops),                 # read G once, read + write the sketch
+        "compress_first": (w.elements * eb + state, flops),               # the cycle's first: the sketch is only written
         "momentum": (w.elements * eb + 2 * state, flops),
         "decompress": (2 * w.elements * eb + state, flops),               # read + write W, read the sketch
         "transfer": (2 * state, transfer_flops),                          # read + write M
@@ -171,6 +172,10 @@ class Rotating:
         self.mark("compress")
         self._next().compress_accumulate(seeds, stream)
 
+    def compress_overwrite(self, seeds, stream=None):
+        self.mark("compress_first")
+        self._next().compress_overwrite(seeds, stream)
+
     def momentum_step(self, beta, seeds, stream=None):
         self.mark("momentum")
         self._next().momentum_step(beta, seeds, stream)
@@ -207,7 +212,7 @@ def make_stepper(w: wl.Workload, acc: Rotating, mom, count: int, base_seed: int,
             if exchange:
                 exchange()
             cyc.apply(LR)
-        return step, f"{w.tau} x compress_accumulate + decompress_apply + zero C"
+        return step, f"{w.tau} x compress (the first overwrites C, the others accumulate) + decompress_apply"
     if w.mode == "momentum":
         st = hostlogic.MomentumState(acc, count, w.beta, w.kappa, base_seed)
         n = [0]
@@ -230,8 +235,8 @@ def make_stepper(w: wl.Workload, acc: Rotating, mom, count: int, base_seed: int,
         if exchange:
             exchange()
         both.apply(LR)
-    return step, (f"{w.tau} x compress_accumulate into C + transfer_axpby (M <- beta M + (1-beta)/tau C A_acc A_mom^T) + "
-                  f"decompress_apply of M + zero C; M resampled every {w.kappa} steps")
+    return step, (f"{w.tau} x compress into C (the first overwrites, the others accumulate) + transfer_axpby "
+                  f"(M <- beta M + (1-beta)/tau C A_acc A_mom^T) + decompress_apply of M; M resampled every {w.kappa} steps")
 
 
 # ------------------------------------------------------------------------------------------ reference arm (CPU oracle)
@@ -446,6 +451,7 @@ def run_flora(args):
     k1 = "compress_pair_kernel" if r > 64 else "compress_tc_kernel"
     k2 = "decompress_pair_kernel" if r > 192 else "decompress_tc_kernel"
     names = {"compress": k1 + " (C += G A^T), one launch over the weight set", "momentum": k1 + " as the momentum update",
+             "compress_first": k1 + " (C <- G A^T, the first compression of a cycle)",
              "momentum_resampled": "gram + apply + compress kernels (Algorithm 2's resampling step)",
              "decompress": ("sketch_to_bf16_kernel + " if r > 64 else "") + k2 + " (W -= lr S A), one launch over the weight set",
              "transfer": "gram + apply kernels (M <- M A_old A_new^T)", "transfer_axpby": "gram + apply kernels (M <- beta M + a C A_acc A_mom^T)"}

@@ -312,6 +312,12 @@ class FloraSet:
         _check(load().flora_set_momentum_step(self._h, beta, _u64_array(seeds), _stream(stream)),
                "flora_set_momentum_step")
 
+    def compress_overwrite(self, seeds: Sequence[int], stream=None) -> None:
+        """C <- G A^T: the first compression of an accumulation cycle, which makes zeroing C beforehand unnecessary
+        (flora_set_momentum_step with beta = 0: the old sketch is neither read nor blended in)."""
+        _check(load().flora_set_momentum_step(self._h, 0.0, _u64_array(seeds), _stream(stream)),
+               "flora_set_momentum_step")
+
     def decompress_apply(self, seeds: Sequence[int], lr: float, scale: float, stream=None) -> None:
         _check(load().flora_set_decompress_apply(self._h, _u64_array(seeds), lr, scale, _stream(stream)),
                "flora_set_decompress_apply")

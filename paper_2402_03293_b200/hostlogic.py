@@ -22,7 +22,8 @@ def _derived(cache: dict, base_seed: int, count: int, epoch: int):
 
 class AccumulationCycle:
     """Algorithm 1: tau compressions into C with one projection per matrix, then one decompression
-    with scale 1/tau; after that C is zeroed and the projection resampled (Section 2.4)."""
+    with scale 1/tau; after that C starts from zero again and the projection is resampled (Section 2.4).
+    The zeroing is folded into the first compression of the next cycle, which overwrites C instead of adding to it."""
 
     def __init__(self, ops, count: int, tau: int, base_seed: int = 0):
         if tau < 1:
@@ -39,7 +40,10 @@ class AccumulationCycle:
         """Compress the gradients currently bound to the set; True when the cycle is full."""
         if self.micro_step >= self.tau:
             raise RuntimeError("cycle is full: call apply() first")
-        self.ops.compress_accumulate(self.seeds(), stream)
+        if self.micro_step == 0:
+            self.ops.compress_overwrite(self.seeds(), stream)         # C <- G A^T: stands for "C <- 0" and the first "C += G A^T"
+        else:
+            self.ops.compress_accumulate(self.seeds(), stream)
         self.micro_step += 1
         return self.micro_step == self.tau
 
@@ -48,7 +52,6 @@ class AccumulationCycle:
         if self.micro_step != self.tau:
             raise RuntimeError("cycle is not full")
         self.ops.decompress_apply(self.seeds(), lr, 1.0 / self.tau, stream)
-        self.ops.zero_state(stream)
         self.epoch += 1
         self.micro_step = 0
 
@@ -118,7 +121,10 @@ class AccumulatedMomentum:
         """Compress the gradients currently bound to `acc`; True when the cycle is full."""
         if self.micro_step >= self.tau:
             raise RuntimeError("cycle is full: call apply() first")
-        self.acc.compress_accumulate(self.acc_seeds(), stream)
+        if self.micro_step == 0:
+            self.acc.compress_overwrite(self.acc_seeds(), stream)     # C <- G A^T: stands for "C <- 0" and the first "C += G A^T"
+        else:
+            self.acc.compress_accumulate(self.acc_seeds(), stream)
         self.micro_step += 1
         return self.micro_step == self.tau
 
@@ -132,7 +138,6 @@ class AccumulatedMomentum:
         cur = self.mom_seeds(self.mom_epoch)
         self.mom.transfer_axpby_from(self.acc, self.acc_seeds(), cur, (1.0 - self.beta) / self.tau, self.beta, stream)
         self.mom.decompress_apply(cur, lr, 1.0, stream)
-        self.acc.zero_state(stream)
         self.acc_epoch += 1
         self.micro_step = 0
         self.t += 1

@@ -64,6 +64,12 @@ class _Mirror:
         for i, rp in self.replays.items():
             rp.compress(self.G()[i], seeds[i])
 
+    def compress_overwrite(self, seeds, stream=None):
+        self.fset.compress_overwrite(seeds, stream)
+        for i, rp in self.replays.items():                        # Algorithm 1 as printed: C <- 0, then C += G A^T
+            rp.S[:] = 0
+            rp.compress(self.G()[i], seeds[i])
+
     def momentum_step(self, beta, seeds, stream=None):
         self.fset.momentum_step(beta, seeds, stream)
         for i, rp in self.replays.items():
@@ -149,7 +155,8 @@ def test_gpt2_xl_set_accumulation_into_momentum_with_outliers():
     w = wl.WORKLOADS["gpt2_xl_set"]
     count, tau = len(w.shapes), 2                    # two of the sixteen micro-steps keep the test short
     W = [wl.weight(w, i, device=DEV, std=0.02) for i in range(count)]
-    C = [torch.zeros(n, w.r, device=DEV) for n, _ in w.shapes]
+    # C holds leftovers (here NaN): a cycle's first compression overwrites it, which stands for Algorithm 1's C <- 0
+    C = [torch.full((n, w.r), float("nan"), device=DEV) for n, _ in w.shapes]
     M = [torch.randn(n, w.r, device=DEV) * 0.01 for n, _ in w.shapes]
     picked = list(range(1, count, 29)) + [count - 1]
     rows = {i: sample_rows(w.shapes[i][0], 8, i) for i in picked}
@@ -174,7 +181,6 @@ def test_gpt2_xl_set_accumulation_into_momentum_with_outliers():
     both.apply(50.0)
     torch.cuda.synchronize()
     _check(rep_m, M, W, w.dtype, "gpt2_xl_set")
-    for i in picked:
-        assert not C[i].any()                        # the cycle ended: C starts the next one at zero
+    assert both.micro_step == 0 and both.t == 1      # the cycle ended; the next one's first compression overwrites C
     acc.close()
     mom.close()

@@ -190,3 +190,39 @@ def test_compression_is_far_closer_to_the_oracle_than_the_tolerance_asks(n, m, r
     print(f"compress {n}x{m} r={r}: normwise {normwise:.2e}, componentwise {componentwise:.2e}")
     assert normwise <= 2e-5
     assert componentwise <= m * 2.0 ** -24
+
+
+@pytest.mark.parametrize("r", [32, 256])
+def test_first_compression_of_a_cycle_overwrites_whatever_the_sketch_held(r):
+    """Algorithm 1 starts a cycle from C = 0; the host classes fold that into the first compression (C <- G A^T).  The
+    result must not depend on what C held before (here NaN and huge values) and must equal zeroing followed by an
+    accumulating compression: to the bit where every row of a sketch has one writer, to rounding where a wide matrix is
+    split along its columns and partial sums are added in whatever order they arrive."""
+    shapes = [(384, 1024), (130, 200), (128, 16384), (1600, 1600)]
+    G = [_g(n, m, 40 + i) for i, (n, m) in enumerate(shapes)]
+    W = [torch.zeros(n, m, device=DEV, dtype=torch.bfloat16) for n, m in shapes]
+    S = [torch.full((n, r), float("nan"), device=DEV) for n, _ in shapes]
+    S[0].fill_(3e38)
+    fset = fb.FloraSet(G, W, S)
+    seeds = [fb.flora_derive_seed(4, i, 0) for i in range(len(shapes))]
+    fset.compress_overwrite(seeds)
+    first = [s.clone() for s in S]
+    fset.zero_state()
+    fset.compress_accumulate(seeds)
+    torch.cuda.synchronize()
+    for i, (n, m) in enumerate(shapes):
+        assert torch.isfinite(first[i]).all(), i
+        assert rel_err(first[i].cpu().numpy(), S[i].cpu().numpy()) <= 1e-6, i
+        assert rel_err(first[i].cpu().numpy(), oracle_compress(G[i], torch.zeros(n, r), seeds[i])) <= TOL["bf16"], i
+    assert torch.equal(first[1], S[1])          # a small matrix has one owner per row in either schedule
+    # the host class uses it: a second cycle starts from the first cycle's leftovers without a zeroing call
+    cyc = hostlogic.AccumulationCycle(fset, len(shapes), tau=2, base_seed=6)
+    for _ in range(2):
+        cyc.accumulate()
+        cyc.accumulate()
+        s_used = cyc.seeds()
+        cyc.apply(0.0)
+    for i, (n, m) in enumerate(shapes):
+        two = oracle_compress(G[i], torch.from_numpy(oracle_compress(G[i], torch.zeros(n, r), s_used[i])), s_used[i])
+        assert rel_err(S[i].cpu().numpy(), two) <= TOL["bf16"], i
+    fset.close()

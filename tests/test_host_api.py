@@ -105,7 +105,8 @@ def test_accumulation_cycle_order_algorithm_1():
     with pytest.raises(RuntimeError):
         cyc.accumulate()
     cyc.apply(0.5)
-    assert [c[0] for c in ops.calls] == ["compress_accumulate"] * 4 + ["decompress_apply", "zero_state"]
+    # the first compression of a cycle overwrites C (zeroing folded into it), the others add
+    assert [c[0] for c in ops.calls] == ["compress_overwrite"] + ["compress_accumulate"] * 3 + ["decompress_apply"]
     assert all(c[1] == s0 for c in ops.calls[:5])                 # one projection for the whole cycle
     assert ops.calls[4][2:] == (0.5, 0.25)                        # arithmetic mean over tau steps
     s1 = cyc.seeds()
@@ -152,7 +153,7 @@ def test_accumulation_feeding_momentum_order():
             both.accumulate()
         both.apply(0.5)
         assert both.acc_seeds() != s_acc                           # a fresh accumulation projection per cycle
-    assert [c[0] for c in acc.calls] == (["compress_accumulate"] * 3 + ["zero_state"]) * 3
+    assert [c[0] for c in acc.calls] == (["compress_overwrite"] + ["compress_accumulate"] * 2) * 3
     names = [c[0] for c in mom.calls]
     # t = 0 resamples (nothing to carry), t = 1 keeps the projection, t = 2 resamples and carries M over first
     assert names == ["transfer_axpby_from", "decompress_apply"] * 2 + ["resample_transfer", "transfer_axpby_from", "decompress_apply"]
