@@ -735,17 +735,33 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
     }
 }
 
-// S <- b S for the listed matrices (those whose rows receive atomic adds from several CTAs); blockIdx.y = list entry.
-__global__ void scale_sketches_kernel(const TcMatrix* __restrict__ mats, const int* __restrict__ ids, int r, float b)
+// S <- b S for the listed matrices (those whose rows receive adds), or for matrix first + blockIdx.y of the table
+// where there is no list; blockIdx.y = list entry.
+__global__ void scale_sketches_kernel(const TcMatrix* __restrict__ mats, const int* __restrict__ ids, int first, int r, float b)
 {
     ptx::grid_launch_dependents();       // the compression kernel that follows may start streaming G right away
-    const TcMatrix* mat = mats + ids[blockIdx.y];
+    const TcMatrix* mat = mats + (ids ? ids[blockIdx.y] : first + (int)blockIdx.y);
+    float* S = mat->S;
     const int64_t total = (int64_t)mat->n * r;
-    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
-        float* p = mat->S + (t / r) * mat->lds + (t % r);
-        *p = (b == 0.0f) ? 0.0f : *p * b;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, nthreads = (int64_t)gridDim.x * blockDim.x;
+    if (mat->lds == r && (reinterpret_cast<uintptr_t>(S) & 15) == 0) {
+        // densely stored, 16-byte aligned: four values per access
+        float4* S4 = reinterpret_cast<float4*>(S);
+        for (int64_t t = tid; t < (total >> 2); t += nthreads) {
+            float4 v = S4[t];
+            v = (b == 0.0f) ? make_float4(0.f, 0.f, 0.f, 0.f) : make_float4(v.x * b, v.y * b, v.z * b, v.w * b);
+            S4[t] = v;
+        }
+        for (int64_t t = (total & ~(int64_t)3) + tid; t < total; t += nthreads) S[t] = (b == 0.0f) ? 0.0f : S[t] * b;
+    } else {
+        for (int64_t row = blockIdx.x; row < mat->n; row += gridDim.x)
+            for (int j = (int)threadIdx.x; j < r; j += (int)blockDim.x) {
+                float* p = S + row * mat->lds + j;
+                *p = (b == 0.0f) ? 0.0f : *p * b;
+            }
     }
 }
+
 
 // bf16 copy of every sketch of the table, n x k_pad with zero padding (the M x K operand of the decompression
 // kernel for ranks above 64); blockIdx.y = matrix.  A thread converts eight neighbouring columns of one row: two
