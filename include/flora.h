@@ -97,7 +97,10 @@ flora_status flora_compress_accumulate(const flora_mat* G, flora_mat* C, uint64_
  * and draws a new seed when a cycle ends (Section 2.4). */
 flora_status flora_decompress_apply(flora_mat* W, const flora_mat* C, uint64_t seed, float lr, float scale, void* stream);
 
-/* Algorithm 2, momentum update:  M <- beta M + (1-beta) G A(seed)^T.   Shapes as for compression. */
+/* Algorithm 2, momentum update:  M <- beta M + (1-beta) G A(seed)^T.   Shapes as for compression.
+ * With beta == 0 the old contents of M are neither read nor blended in (they may be uninitialised, NaN included):
+ * M <- G A(seed)^T.  That is also the first compression of an accumulation cycle of Algorithm 1 with its
+ * "C <- 0" folded in. */
 flora_status flora_momentum_step(const flora_mat* G, flora_mat* M, float beta, uint64_t seed, void* stream);
 
 /* Algorithm 2, resampling branch:  M <- M A(seed_old) A(seed_new)^T, evaluated as M (A_old A_new^T).
@@ -169,6 +172,7 @@ flora_status flora_set_rebind_gradients(flora_set* set, const flora_mat* G, void
 
 /* seeds: host array of `count` 64-bit seeds, one per matrix (copied before the call returns). */
 flora_status flora_set_compress_accumulate(flora_set* set, const uint64_t* seeds, void* stream);
+/* (beta == 0 overwrites the sketches, as for flora_momentum_step) */
 flora_status flora_set_momentum_step(flora_set* set, float beta, const uint64_t* seeds, void* stream);
 flora_status flora_set_decompress_apply(flora_set* set, const uint64_t* seeds, float lr, float scale, void* stream);
 flora_status flora_set_resample_transfer(flora_set* set, const uint64_t* seeds_old, const uint64_t* seeds_new, void* stream);
