@@ -376,7 +376,8 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
             const int sb = k & 1;
             ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_empty[sb]), (((uint32_t)k >> 1) & 1u) ^ 1u, abort);
             if (!ok) break;
-            k2_generate_slab<true>(slab0 + sb * slab_bytes, slab_block, kchunks, 64, item.col0 + 64 * (int)half, r, key, scale, g, 32 * K2P_GEN_WARPS);
+            if (item.tiles > 0)         // (an empty item pads a CTA's list: its slab is never read)
+                k2_generate_slab<true>(slab0 + sb * slab_bytes, slab_block, kchunks, 64, item.col0 + 64 * (int)half, r, key, scale, g, 32 * K2P_GEN_WARPS);
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {

@@ -652,8 +652,9 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
                 // share of the slab alongside the generator warps.
                 ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_empty[0]), (((nslabs == 2 ? (k >> 1) : k) & 1) ^ 1), abort);
                 if (!ok) break;
-                k2_generate_slab<BF16S>(slab0, slab_block, kchunks, bn, item.col0, r, make_key(seeds.s[item.mat - seed_base]), scale,
-                                        32 * GW + helper, 32 * (GW + K2_HELPER_WARPS));
+                if (item.tiles > 0)     // (an empty item pads a CTA's list: its slab is never read)
+                    k2_generate_slab<BF16S>(slab0, slab_block, kchunks, bn, item.col0, r, make_key(seeds.s[item.mat - seed_base]), scale,
+                                            32 * GW + helper, 32 * (GW + K2_HELPER_WARPS));
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->slab_help));
@@ -720,8 +721,9 @@ decompress_tc_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restrict
             if (!ok) break;
             const uint32_t slab = slab0 + sb * slab_bytes;
             // the first slab (every slab, with a single buffer) is shared with the combine warps
-            k2_generate_slab<BF16S>(slab, slab_block, kchunks, bn, item.col0, r, key, scale, g,
-                                    (k == 0 || nslabs == 1) ? 32 * (GW + K2_HELPER_WARPS) : 32 * GW);
+            if (item.tiles > 0)
+                k2_generate_slab<BF16S>(slab, slab_block, kchunks, bn, item.col0, r, key, scale, g,
+                                        (k == 0 || nslabs == 1) ? 32 * (GW + K2_HELPER_WARPS) : 32 * GW);
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->slab_full[sb]));

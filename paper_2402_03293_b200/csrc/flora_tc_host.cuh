@@ -686,10 +686,94 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
             set.h_k2 = cand;
         }
     }
+    // A set with few slabs per CTA (one matrix, say: 86 slabs for 74 pairs) leaves the CTAs unevenly loaded however the
+    // slabs are cut into runs.  Candidate: every CTA (pair) gets an equal, contiguous share of the row-tile steps of all
+    // slabs in order, cut wherever the share ends.  A share is one to three pieces of neighbouring slabs, taken largest
+    // first so that the generation of the next piece's slab hides behind the streaming of the current one.  The kernels
+    // hand out items round-robin, so piece j of CTA c sits at index j * G + c; a CTA with fewer pieces than the others
+    // gets an empty item (no tiles: nothing is generated or streamed for it) at the end.
+    bool balanced = false;
+    int balanced_grid = 0;
+    if (!fixed_run && W.size() <= (size_t)SEEDS_PER_LAUNCH) {
+        const int per_step = pair ? 2 : 1;
+        int64_t total = 0;
+        for (const auto& w : W)
+            if (w.rows > 0 && w.cols > 0) total += (((w.rows + 127) / 128 + per_step - 1) / per_step) * ((w.cols + bn - 1) / bn);
+        const int G = (int)std::min<int64_t>(grid_max, total);
+        if (G > 0) {
+            std::vector<std::vector<K2Item>> share((size_t)G);
+            int64_t pos = 0;
+            int c = 0;
+            for (size_t i = 0; i < W.size(); ++i) {
+                const auto& w = W[i];
+                if (w.rows == 0 || w.cols == 0) continue;
+                const int64_t rtiles = (w.rows + 127) / 128, steps = (rtiles + per_step - 1) / per_step, nsl = (w.cols + bn - 1) / bn;
+                for (int64_t sl = 0; sl < nsl; ++sl) {
+                    int64_t s0 = 0;
+                    while (s0 < steps) {
+                        while (c + 1 < G && pos >= ((int64_t)(c + 1) * total + G - 1) / G) ++c;
+                        const int64_t end_c = c + 1 < G ? ((int64_t)(c + 1) * total + G - 1) / G : total;
+                        const int64_t take = std::min<int64_t>(steps - s0, end_c - pos);
+                        K2Item it;
+                        it.mat = (int)i;
+                        it.col0 = (int)(sl * bn);
+                        it.row0 = (int)(s0 * per_step * 128);
+                        it.tiles = (int)std::min<int64_t>(take * per_step, rtiles - s0 * per_step);
+                        share[(size_t)c].push_back(it);
+                        pos += take;
+                        s0 += take;
+                    }
+                }
+            }
+            size_t most = 0;
+            double span = 0.0;
+            for (auto& sh : share) {
+                std::stable_sort(sh.begin(), sh.end(), [](const K2Item& x, const K2Item& y) { return x.tiles > y.tiles; });
+                most = std::max(most, sh.size());
+                // the slab of piece k + 1 is generated while piece k streams (the first one is charged like any item of
+                // the run-based candidates, which the comparison is with)
+                double t = 0.0;
+                const double gen = pair_f * t_slab;
+                for (size_t k = 0; k < sh.size(); ++k) {
+                    const double stream = (pair ? (sh[k].tiles + 1) / 2 : sh[k].tiles) * t_tile;
+                    if (nslabs == 1) {
+                        t += K2_EXPOSED_ONE_SLAB * gen + stream + K2_ITEM_OVERHEAD_US;
+                    } else {
+                        const double next_gen = k + 1 < sh.size() ? gen : 0.0;
+                        t += stream + K2_OVERLAP_PENALTY * std::min(next_gen, stream) + std::max(0.0, next_gen - stream) + K2_ITEM_OVERHEAD_US;
+                    }
+                }
+                span = std::max(span, t);
+            }
+            if (span < best * 0.97) {
+                best = span;
+                balanced = true;
+                balanced_grid = G;
+                set.h_k2.assign(most * (size_t)G, K2Item());
+                for (int q = 0; q < G; ++q)
+                    for (size_t j = 0; j < most; ++j) {
+                        K2Item& slot = set.h_k2[j * (size_t)G + (size_t)q];
+                        if (j < share[(size_t)q].size()) {
+                            slot = share[(size_t)q][j];
+                        } else {
+                            slot.mat = share[(size_t)q][0].mat;
+                            slot.col0 = 0;
+                            slot.row0 = 0;
+                            slot.tiles = 0;
+                        }
+                    }
+            }
+        }
+    }
     // launches cover at most SEEDS_PER_LAUNCH consecutive matrices; inside a launch the largest items go first
     set.k2_launch_begin.clear();
     set.k2_launch_first_mat.clear();
     size_t u0 = 0;
+    if (balanced) {                     // one launch over all matrices (there are at most SEEDS_PER_LAUNCH), order as laid out
+        set.k2_launch_begin.push_back(0);
+        set.k2_launch_first_mat.push_back(0);
+        u0 = set.h_k2.size();
+    }
     while (u0 < set.h_k2.size()) {
         size_t u1 = u0;
         while (u1 < set.h_k2.size() && set.h_k2[u1].mat < set.h_k2[u0].mat + SEEDS_PER_LAUNCH) ++u1;
@@ -699,7 +783,7 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
         u0 = u1;
     }
     set.k2_launch_begin.push_back((int)set.h_k2.size());
-    set.k2_grid_max = grid_max;
+    set.k2_grid_max = balanced ? balanced_grid : grid_max;
 }
 
 inline void tc_set_free_stream(TcSet& s, cudaStream_t st)
