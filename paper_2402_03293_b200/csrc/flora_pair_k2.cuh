@@ -34,7 +34,7 @@ constexpr int K2P_ACCS = 4;           // accumulators in tensor memory: two per 
 
 struct K2PairSmem {
     uint64_t w_full[K2_MAX_SLOTS], out_ready[K2_MAX_SLOTS];
-    uint64_t c_full[K2_MAX_CSTAGES], c_empty[K2_MAX_CSTAGES], acc_full[K2P_ACCS], acc_empty[K2P_ACCS], slab_full[2], slab_empty[2];
+    uint64_t c_full[K2_MAX_CSTAGES], c_empty[K2_MAX_CSTAGES], acc_full[K2P_ACCS], acc_empty[K2P_ACCS], slab_full[2], slab_empty[2], slab_help;
     uint32_t tmem_base;
     int abort;
 };
@@ -87,6 +87,7 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
             ptx::mbar_init(ptx::smem_addr(&ctl->slab_full[s]), 2 * K2P_GEN_WARPS);  // the generator warps of both CTAs (leader's barrier)
             ptx::mbar_init(ptx::smem_addr(&ctl->slab_empty[s]), 2);                 // both MMA threads are done with the slab
         }
+        ptx::mbar_init(ptx::smem_addr(&ctl->slab_help), 16);    // the combine warps of both CTAs have written their share of the first slab
         ctl->abort = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
@@ -199,6 +200,9 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
             cur_init(cs[1], 1);
             RingPos prs[2];
             bool ok = true;
+            // the bf16 copy of the sketches is written by the kernel before this one, which lets this one start early
+            // (programmatic dependent launch): nothing else here reads what that kernel writes
+            ptx::grid_dependency_wait();
             while (ok && (cs[0].it < n_items || cs[1].it < n_items)) {
                 for (int kc = 0; kc < kchunks && ok; ++kc) {
 #pragma unroll
@@ -253,6 +257,7 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
                 const int sb = c.k & 1;
                 const uint64_t desc_slab = ptx::umma_desc_k_sw128(slab0 + sb * slab_bytes);
                 ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_full[sb]), (uint32_t)(c.k >> 1) & 1u, abort);     // both halves of the slab are written
+                if (c.k == 0 && ok) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_help), 0u, abort);              // ... the combine warps' share of the first one too
                 for (; c.p < c.n && ok; c.p += 2, gt += 2) {
                     const int a = gt & (K2P_ACCS - 1);
                     const uint32_t acc_addr = tmem + (uint32_t)a * K2P_BN;
@@ -309,6 +314,21 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
         RingPos pw;
         int gt = 0;
         bool ok = true;
+        if (cluster < n_items) {
+            // nothing to combine yet: write a share of the first slab alongside the generator warps
+            const K2Item first = items[cluster];
+            const int helper = ((warp >= 8 ? warp - 4 : warp - 2) << 5) + lane;           // 0 .. 255
+            if (first.tiles > 0)
+                k2_generate_slab<true>(slab0, slab_block, kchunks, 64, first.col0 + 64 * (int)half, r, make_key(seeds.s[first.mat - seed_base]), scale,
+                                       32 * K2P_GEN_WARPS + helper, 32 * (K2P_GEN_WARPS + 8));
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                const uint32_t hbar = ptx::smem_addr(&ctl->slab_help);
+                if (half == 0) ptx::mbar_arrive(hbar);
+                else ptx::mbar_arrive_cluster_release(ptx::map_to_cta(hbar, 0u));
+            }
+        }
         for (int it = cluster; it < n_items && ok; it += clusters) {
             const K2Item item = items[it];
             const int live_chunks = min(2, (mats[item.mat].m - item.col0 + 63) >> 6) << 2;     // 16-column chunks that hold columns of W
@@ -377,7 +397,8 @@ decompress_pair_kernel(const TcMatrix* __restrict__ mats, const K2Item* __restri
             ok = ptx::mbar_wait(ptx::smem_addr(&ctl->slab_empty[sb]), (((uint32_t)k >> 1) & 1u) ^ 1u, abort);
             if (!ok) break;
             if (item.tiles > 0)         // (an empty item pads a CTA's list: its slab is never read)
-                k2_generate_slab<true>(slab0 + sb * slab_bytes, slab_block, kchunks, 64, item.col0 + 64 * (int)half, r, key, scale, g, 32 * K2P_GEN_WARPS);
+                k2_generate_slab<true>(slab0 + sb * slab_bytes, slab_block, kchunks, 64, item.col0 + 64 * (int)half, r, key, scale, g,
+                                       k == 0 ? 32 * (K2P_GEN_WARPS + 8) : 32 * K2P_GEN_WARPS);      // the first slab is shared with the combine warps
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {

@@ -771,6 +771,7 @@ __global__ void scale_sketches_kernel(const TcMatrix* __restrict__ mats, const i
 // threads covers 2048 / k_pad rows at a time.
 __global__ void __launch_bounds__(256) sketch_to_bf16_kernel(const TcMatrix* __restrict__ mats, int r, int k_pad)
 {
+    ptx::grid_launch_dependents();       // the decompression kernel that follows may set up and generate its first slabs meanwhile
     const TcMatrix* mat = mats + blockIdx.y;
     const int groups = k_pad >> 3;                        // 8-column groups per row: 8, 16, 24 or 32
     const int rows_per_block = 256 / groups;

@@ -1134,13 +1134,15 @@ inline flora_status tc_set_decompress(TcSet& set, const uint64_t* seeds, float s
             cfg.blockDim = dim3((unsigned)K2P_THREADS);
             cfg.dynamicSmemBytes = set.k2_smem;
             cfg.stream = st;
-            cudaLaunchAttribute attr[1];
+            cudaLaunchAttribute attr[2];
             attr[0].id = cudaLaunchAttributeClusterDimension;
             attr[0].val.clusterDim.x = 2;
             attr[0].val.clusterDim.y = 1;
             attr[0].val.clusterDim.z = 1;
+            attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // the kernel's sketch loader waits for its predecessor itself
+            attr[1].val.programmaticStreamSerializationAllowed = 1;
             cfg.attrs = attr;
-            cfg.numAttrs = 1;
+            cfg.numAttrs = 2;
             const TcMatrix* mats = set.d_mats;
             const K2Item* items = set.d_k2 + begin;
             if (cudaLaunchKernelEx(&cfg, decompress_pair_kernel, mats, items, end - begin, table, seed_base, r, scale, step, set.slots, set.cstages) !=
