@@ -449,7 +449,7 @@ def run_flora(args):
     costs = op_costs(w, r)
     hbm, tf, src = measured_peaks()
     k1 = "compress_pair_kernel" if r > 64 else "compress_tc_kernel"
-    k2 = "decompress_pair_kernel" if r > 192 else "decompress_tc_kernel"
+    k2 = "decompress_pair_kernel" if r > 128 else "decompress_tc_kernel"
     names = {"compress": k1 + " (C += G A^T), one launch over the weight set", "momentum": k1 + " as the momentum update",
              "compress_first": k1 + " (C <- G A^T, the first compression of a cycle)",
              "momentum_resampled": "gram + apply + compress kernels (Algorithm 2's resampling step)",

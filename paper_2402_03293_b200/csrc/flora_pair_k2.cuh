@@ -1,17 +1,19 @@
-// Decompression fused with the update for ranks above 192 on CTA pairs (tcgen05.mma.cta_group::2):  W <- W - step * S A.
+// Decompression fused with the update for ranks above 128 on CTA pairs (tcgen05.mma.cta_group::2):  W <- W - step * S A.
 //
 // Same structure as decompress_tc_kernel (a slab of 128 columns of A stays resident while the row tiles of W stream
 // past it), with two CTAs working on one slab: an MMA multiplies the 128 rows of the sketch tile of either CTA
 // (M = 256) with the slab, of which each CTA generates and holds only the 64 columns that the instruction takes
 // from its shared memory (the N x K operand is split over the pair).  Half a slab is 32 KB at r = 256, so two
 // buffers fit and the slab of the next item is generated while the current item streams, which a single CTA
-// cannot do above r = 192.  The pair takes the row tiles of an item in turn (the leader the even ones), so an item
-// streams in half the time and each CTA generates half as much per item.  Each CTA loads, combines and stores its
-// own W tiles (two slots; the tile that will follow a tile in its slot is asked into L2 meanwhile).  The leader issues the MMAs for both, from two threads: a thread gets an MMA accepted only about every
-// hundred cycles, and with sixteen of them and five commits per tile iteration one thread alone sets the pace of the
-// kernel.  The two take the tile iterations in turn, each with two of the four accumulators and its own ring of sketch
-// chunks, filled in step with the other's, and each learns from a relay thread of the follower that the follower's
-// chunks have landed.
+// cannot do above r = 192 (below that the pair is faster as well, down to r = 129: measured).  The pair takes the
+// row tiles of an item in turn (the leader the even ones), so an item streams in half the time and each CTA
+// generates half as much per item.  Each CTA loads, combines and stores its own W tiles (two slots or more; the
+// tile that will follow a tile in its slot is asked into L2 meanwhile).  The leader issues the MMAs for both, from
+// two threads: a thread gets an MMA accepted only about every hundred cycles, and with sixteen of them and five
+// commits per tile iteration one thread alone sets the pace of the kernel.  The two take the tile iterations in
+// turn, each with two of the four accumulators and its own ring of sketch chunks, filled in step with the other's,
+// and each learns from a relay thread of the follower that the follower's chunks have landed.  The combine warps,
+// idle until the first accumulator is full, share the generation of the pair's first slab.
 // The sketch is read from its bf16 copy (see sketch_to_bf16_kernel).  All waits are bounded.
 #pragma once
 #include <cuda.h>

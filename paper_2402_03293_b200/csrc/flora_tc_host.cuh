@@ -610,10 +610,12 @@ inline void plan_decompress(TcSet& set, const std::vector<flora_mat>& W, int r)
     set.k2_nslabs = nslabs;
     set.k2_smem = nslabs * slab_bytes + (size_t)cstages * S_CHUNK_BYTES + (size_t)slots * slot + sizeof(K2Smem) + 1024;
     int grid_max = sm_count() * per_sm;
-    // Ranks whose slab leaves one CTA room for a single buffer run on CTA pairs: each CTA holds half of a 128-column slab (two buffers of kchunks x 8 KB), the
+    // Ranks above 128 run on CTA pairs: each CTA holds half of a 128-column slab (two buffers of kchunks x 8 KB), the
     // sketch chunks of its own tiles (as many stages as fit beside two W tiles, at most two tiles' worth) and its W tiles.
-    // (where one CTA has room for two slab buffers itself, up to r = 192, it is the faster of the two: measured)
-    const bool pair = bf16s && tune_knob("FLORA_K2_PAIR", nslabs == 1 ? 1 : 0, 0, 1) != 0;
+    // Above r = 192 one CTA has room for a single slab buffer only; from r = 129 to 192 it has room for two, and the pair
+    // is still the faster (config 5's set at r = 192: 1335 against 1447 us; one 4096 x 11008 matrix: 54 against 58 us).
+    // Up to r = 128 one CTA per SM wins on sets (1087 against 1453 us).
+    const bool pair = bf16s && tune_knob("FLORA_K2_PAIR", kchunks >= 3 ? 1 : 0, 0, 1) != 0;
     set.k2_pair = pair;
     if (pair) {
         const size_t half_slab = (size_t)kchunks * 64 * 128, pslot = 2 * (size_t)W_BOX_BYTES;
