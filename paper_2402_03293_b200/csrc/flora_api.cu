@@ -366,12 +366,13 @@ flora_status flora_set_rebind_gradients(flora_set* set, const flora_mat* G, void
     return FLORA_OK;
 }
 
-static flora_status set_compress(flora_set* set, const uint64_t* seeds, float a, float b, void* stream)
+// behind_own_transfer: the kernel before this call on the stream is the library's own transfer, which does not touch G
+static flora_status set_compress(flora_set* set, const uint64_t* seeds, float a, float b, void* stream, bool behind_own_transfer = false)
 {
     if (!set || !seeds) return FLORA_ERR_NULL;
     if (!set->has_G) return FLORA_ERR_UNSUPPORTED;
     if (set->tc.compress_ready && g_force_path.load() != 1)
-        return tc_set_compress(set->tc, seeds, a, b, as_stream(stream), g_launches);
+        return tc_set_compress(set->tc, seeds, a, b, as_stream(stream), g_launches, behind_own_transfer);
     for (size_t i = 0; i < set->G.size(); ++i) {
         if (set->G[i].rows == 0) continue;
         flora_status st = simt_compress(&set->G[i], &set->S[i], seeds[i], a, b, as_stream(stream));
@@ -406,8 +407,9 @@ flora_status flora_set_decompress_apply(flora_set* set, const uint64_t* seeds, f
 
 // dst.S[i] <- b dst.S[i] + a src[i] (A(old_i) A(new_i)^T) for every matrix of the set `dst`.
 static flora_status set_transfer(flora_set* set, const std::vector<flora_mat>& src, const TcMatrix* src_mats, const uint64_t* seeds_old,
-                                 const uint64_t* seeds_new, float a, float b, void* stream)
+                                 const uint64_t* seeds_new, float a, float b, void* stream, void** release_later = nullptr)
 {
+    if (release_later) *release_later = nullptr;
     if (!set || !seeds_old || !seeds_new) return FLORA_ERR_NULL;
     const std::vector<flora_mat>& big = set->has_G ? set->G : set->W;
     const int r = set->r;
@@ -423,7 +425,7 @@ static flora_status set_transfer(flora_set* set, const std::vector<flora_mat>& s
             jobs.push_back(GramJob{nullptr, (float*)set->S[i].data, (const float*)src[i].data, set->S[i].ld, src[i].ld,
                                    (int32_t)set->S[i].rows, (int32_t)big[i].cols, seeds_old[i], seeds_new[i], (int32_t)i, 0});
         }
-        return transfer_tc(jobs, r, a, b, as_stream(stream), g_launches, set->tc.d_mats, src_mats);
+        return transfer_tc(jobs, r, a, b, as_stream(stream), g_launches, set->tc.d_mats, src_mats, nullptr, release_later);
     }
     if (scratch_alloc((void**)&T, sizeof(float) * r * r, as_stream(stream)) != cudaSuccess) {
         cudaGetLastError();
@@ -458,9 +460,13 @@ flora_status flora_set_momentum_step_resampled(flora_set* set, float beta, const
 {
     if (!set || !seeds_old || !seeds_new) return FLORA_ERR_NULL;
     if (!set->has_G) return FLORA_ERR_UNSUPPORTED;
-    flora_status st = set_transfer(set, set->S, set->tc.d_mats, seeds_old, seeds_new, beta, 0.0f, stream);
-    if (st) return st;
-    return set_compress(set, seeds_new, 1.0f - beta, 1.0f, stream);
+    // the compression goes right behind the transfer's last kernel and starts while that one still runs (it waits itself
+    // before it touches a sketch); the transfer's scratch is handed back after it has been launched
+    void* scratch = nullptr;
+    flora_status st = set_transfer(set, set->S, set->tc.d_mats, seeds_old, seeds_new, beta, 0.0f, stream, &scratch);
+    if (st == FLORA_OK) st = set_compress(set, seeds_new, 1.0f - beta, 1.0f, stream, scratch != nullptr);
+    if (scratch && cudaFreeAsync(scratch, as_stream(stream)) != cudaSuccess && st == FLORA_OK) st = FLORA_ERR_CUDA;
+    return st;
 }
 
 flora_status flora_set_zero_state(flora_set* set, void* stream)

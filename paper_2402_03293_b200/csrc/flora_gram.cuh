@@ -381,6 +381,9 @@ apply_tc_kernel(const GramJob* __restrict__ jobs, const TcMatrix* __restrict__ d
                 const ApplyUnit* __restrict__ units, const int* __restrict__ slot_begin, const __grid_constant__ ApplySingle single, int per_cluster,
                 int r, float aa, float bb)
 {
+    // A kernel launched behind this one with the programmatic-serialization attribute may start now (the compression of
+    // a resampling step does: it streams G, which this kernel does not touch, and waits itself before it reads a sketch).
+    ptx::grid_launch_dependents();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
     const int N = (r + 15) & ~15, n_half = N >> 1, kchunks = (r + 31) >> 5;
@@ -658,8 +661,12 @@ apply_tc_kernel(const GramJob* __restrict__ jobs, const TcMatrix* __restrict__ d
 // table upload, the two kernels, the release of the scratch.  A single matrix: only the r x r scratch; the job
 // travels as a kernel parameter.  `jobs` come without T; it is assigned here.
 inline flora_status transfer_tc(std::vector<GramJob>& jobs, int r, float a, float b, cudaStream_t st, std::atomic<uint64_t>& launches,
-                                const TcMatrix* d_dst_mats = nullptr, const TcMatrix* d_src_mats = nullptr, float* static_T = nullptr)
+                                const TcMatrix* d_dst_mats = nullptr, const TcMatrix* d_src_mats = nullptr, float* static_T = nullptr,
+                                void** release_later = nullptr)
 {
+    // release_later: the caller frees the call's scratch (stream-ordered) itself, after it has put more work behind the
+    // last kernel; nothing then stands between that kernel and the caller's next launch
+    if (release_later) *release_later = nullptr;
     if (jobs.empty()) return FLORA_OK;
     int sms = 148, dev = 0;
     cudaGetDevice(&dev);
@@ -830,7 +837,10 @@ inline flora_status transfer_tc(std::vector<GramJob>& jobs, int r, float a, floa
         }
     }
     if (!ok || cudaPeekAtLastError() != cudaSuccess) rc = FLORA_ERR_CUDA;
-    if (!static_T && cudaFreeAsync(buf, st) != cudaSuccess && rc == FLORA_OK) rc = FLORA_ERR_CUDA;
+    if (!static_T) {
+        if (release_later) *release_later = buf;
+        else if (cudaFreeAsync(buf, st) != cudaSuccess && rc == FLORA_OK) rc = FLORA_ERR_CUDA;
+    }
     return rc;
 }
 

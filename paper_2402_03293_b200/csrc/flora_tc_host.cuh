@@ -948,12 +948,14 @@ inline unsigned helper_blocks(const TcSet& set)
     return (unsigned)std::min<int64_t>(1024, (most + 1023) / 1024);
 }
 
+// behind_own_kernel: the kernel before this call on the stream is one of the library's own that does not touch G and lets
+// its dependents start early (the transfer's apply kernel): only the write-out of the compression waits for it.
 inline flora_status tc_set_compress(TcSet& set, const uint64_t* seeds, float a, float b, cudaStream_t st,
-                                    std::atomic<uint64_t>& launches)
+                                    std::atomic<uint64_t>& launches, bool behind_own_kernel = false)
 {
     const int r = set.r;
     const float scale = 1.0f / sqrtf((float)r);
-    int late_wait = 0;
+    int late_wait = behind_own_kernel ? tune_knob("FLORA_PDL", 1, 0, 1) : 0;
     const bool pair = set.k1_pair;
     // The pair kernel blends an old sketch in (S <- b S + a G A^T) faster as a scaling pass followed by its reducing
     // write-out than by reading the old values back in its epilogue, as long as the sketches are few enough to stay in
