@@ -243,9 +243,9 @@ def make_stepper(w: wl.Workload, acc: Rotating, mom, count: int, base_seed: int,
 class OracleSample:
     """The workload's step on a sample of rows of the first transformer block's matrices, on the CPU oracle."""
 
-    def __init__(self, w: wl.Workload, r: int, rows: int):
+    def __init__(self, w: wl.Workload, r: int, rows: int, lr: float = LR):
         import numpy as np
-        self.np, self.w, self.r = np, w, r
+        self.np, self.w, self.r, self.lr = np, w, r, lr
         block = 4 if "gpt2" in w.name else (7 if "t5" in w.name else 1)
         self.ids = list(range(min(block, len(w.shapes))))
         self.rows = [min(rows, w.shapes[i][0]) for i in self.ids]
@@ -270,7 +270,7 @@ class OracleSample:
                 self.C[j][:] = 0
                 for k in range(w.tau):
                     orc.compress_accumulate(self.G[k % len(self.G)][j], A, self.C[j])
-                orc.decompress_apply(self.W[j], self.C[j], A, LR, 1.0 / w.tau)
+                orc.decompress_apply(self.W[j], self.C[j], A, self.lr, 1.0 / w.tau)
             elif w.mode == "momentum":
                 epoch = t // w.kappa if w.kappa else 0
                 A = orc.projection(1000 * epoch + i, r, m, w.dtype)
@@ -281,7 +281,7 @@ class OracleSample:
                     orc.momentum_step_resampled(self.G[0][j], A_old, A, w.beta, self.M[j])
                 else:
                     orc.momentum_step(self.G[0][j], A, w.beta, self.M[j])
-                orc.decompress_apply(self.W[j], self.M[j], A, LR, 1.0)
+                orc.decompress_apply(self.W[j], self.M[j], A, self.lr, 1.0)
             else:
                 A_acc = orc.projection(1000 * t + i, r, m, w.dtype)
                 A_mom = orc.projection(7_000_000 + i, r, m, w.dtype)
@@ -289,13 +289,78 @@ class OracleSample:
                 for k in range(w.tau):
                     orc.compress_accumulate(self.G[k % len(self.G)][j], A_acc, self.C[j])
                 orc.transfer_axpby(self.M[j], self.C[j], A_acc, A_mom, (1.0 - w.beta) / w.tau, w.beta)
-                orc.decompress_apply(self.W[j], self.M[j], A_mom, LR, 1.0)
+                orc.decompress_apply(self.W[j], self.M[j], A_mom, self.lr, 1.0)
         self.t += 1
         return time.perf_counter() - t0
 
     def describe(self):
         names = ", ".join(f"{n} of {self.w.shapes[i][0]} rows of a {self.w.shapes[i][0]}x{self.w.shapes[i][1]} matrix" for i, n in zip(self.ids, self.rows))
         return f"the whole step on the first rows of one transformer block's matrices ({names}); GB/s is per row processed, so it extrapolates linearly"
+
+
+def sample_parity(w: wl.Workload, r: int, fb, rows: int = 48) -> dict:
+    """The first step of the workload on a few rows of one transformer block's matrices, on the GPU path and on the
+    oracle (part of the cpu_baseline leg): normwise maximum error of the compressed state and of the weight update."""
+    import numpy as np
+    from oracle import flora_oracle as orc
+    dev = "cuda"
+
+    def to_gpu(a):                                   # stored bytes -> device tensor (bf16 travels as its bit patterns)
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16).copy()).to(dev).view(torch.bfloat16)
+        return torch.from_numpy(a.copy()).to(dev)
+
+    def vals(a):
+        return (orc.bf16_bits_to_f32(a) if a.dtype == np.uint16 else a).astype(np.float64)
+
+    def err(x, y):
+        return float(np.max(np.abs(x - y)) / max(float(np.max(np.abs(y))), 1e-300))
+
+    # a step size that makes the update about half as large as the weights, so that its error is not hidden below the
+    # bf16 spacing of W (the benchmark's own step is far smaller): found from one oracle step with step size 1
+    probe = OracleSample(w, r, rows, 1.0)
+    before = [vals(x) for x in probe.W]
+    probe.step()
+    moved = max(float(np.max(np.abs(vals(x) - b))) for x, b in zip(probe.W, before))
+    lr = 0.5 * max(float(np.max(np.abs(b))) for b in before) / max(moved, 1e-30)
+    ref = OracleSample(w, r, rows, lr)
+    G = [[to_gpu(g) for g in gs] for gs in ref.G]
+    W0 = [vals(x) for x in ref.W]
+    W = [to_gpu(x) for x in ref.W]
+    C = [torch.full((n, r), float("nan"), device=dev) for n in ref.rows]      # a cycle's first compression overwrites
+    M = [torch.zeros(n, r, device=dev) for n in ref.rows]
+    ref.step()
+    ids = ref.ids                                    # the oracle sample's seeds at t = 0 are the matrix numbers
+    if w.mode == "accumulate":
+        sets = [fb.FloraSet(G[0], W, C)]
+        for k in range(w.tau):
+            sets[0].rebind_gradients(G[k % len(G)])
+            (sets[0].compress_overwrite if k == 0 else sets[0].compress_accumulate)(ids)
+        sets[0].decompress_apply(ids, lr, 1.0 / w.tau)
+        state, state_ref = C, ref.C
+    elif w.mode == "momentum":
+        sets = [fb.FloraSet(G[0], W, M)]
+        sets[0].momentum_step(w.beta, ids)
+        sets[0].decompress_apply(ids, lr, 1.0)
+        state, state_ref = M, ref.M
+    else:
+        acc, mom = fb.FloraSet(G[0], None, C), fb.FloraSet(None, W, M)
+        sets = [acc, mom]
+        s_mom = [7_000_000 + i for i in ids]
+        for k in range(w.tau):
+            acc.rebind_gradients(G[k % len(G)])
+            (acc.compress_overwrite if k == 0 else acc.compress_accumulate)(ids)
+        mom.transfer_axpby_from(acc, ids, s_mom, (1.0 - w.beta) / w.tau, w.beta)
+        mom.decompress_apply(s_mom, lr, 1.0)
+        state, state_ref = M, ref.M
+    torch.cuda.synchronize()
+    e_state = max(err(s_.cpu().numpy().astype(np.float64), sr.astype(np.float64)) for s_, sr in zip(state, state_ref))
+    e_upd = max(err(W[j].float().cpu().numpy().astype(np.float64) - W0[j], vals(ref.W[j]) - W0[j]) for j in range(len(ids)))
+    for s_ in sets:
+        s_.close()
+    return {"state_max_rel_err": e_state, "weight_update_max_rel_err": e_upd, "tolerance": 2e-2, "step_size": lr,
+            "what": f"first step on {rows} rows of each matrix of one transformer block: GPU path against the CPU oracle, "
+                    "max |x - ref| / max |ref| of the compressed state and of W - W0, at a step size that moves the weights by half their size"}
 
 
 def sized_oracle_sample(w: wl.Workload, r: int, seconds_per_step: float) -> OracleSample:
@@ -501,7 +566,7 @@ def run_flora(args):
            "d2h_bytes_per_step": w.elements * w.elem_bytes, "steps": e2e_steps,
            "api": "flora_set_upload_gradients + the step's set calls + flora_set_read_weights_to_host, pinned host buffers"}
 
-    cpu_baseline = None
+    cpu_baseline, parity = None, None
     if rank == 0 and world == 1:
         from oracle import flora_oracle as orc
         sample = sized_oracle_sample(w, r, 4.0)
@@ -511,6 +576,7 @@ def run_flora(args):
             n_steps += 1
         cpu_baseline = {"value": sample.grad_bytes() * n_steps / total_t / 1e9, "unit": "GB/s", "cores": orc.max_threads(), "kind": "oracle",
                         "sample": f"{n_steps} step(s), {total_t:.1f} s wall: " + sample.describe()}
+        parity = sample_parity(w, r, fb)
 
     if rank == 0:
         line = {
@@ -522,7 +588,7 @@ def run_flora(args):
                        "l2": f"inputs larger than L2: {n_sets} rotating gradient sets of {grad_set_bytes / 1e9:.2f} GB, a different one per compression",
                        "timed": f"{len(blocks)} block(s) of {args.steps} steps, {spent:.2f} s of device time; value is the median block",
                        "multi_gpu": "data-parallel ranks, all-reduce of the sketches" if exchange else "independent replicas, no collective"},
-            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches_per_block), "clocks": clocks,
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "parity": parity, "e2e": e2e, "gpu_launches": int(launches_per_block), "clocks": clocks,
             "ms_x_mhz_per_step": (ms / args.steps) * clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None,
         }
         print(json.dumps(line), flush=True)
