@@ -214,9 +214,6 @@ constexpr double K1_GENERATION_PER_RANK = 0.045;
 constexpr double K2_SM_BYTES_PER_US = 60e3;
 constexpr double K2_VALUES_PER_US_8_WARPS = 2000.0, K2_VALUES_PER_US_FEWER = 1300.0;
 constexpr double K2_EXPOSED_ONE_SLAB = 0.55, K2_OVERLAP_PENALTY = 0.35, K2_ITEM_OVERHEAD_US = 0.2;
-// Values of A that the generator warps of one SM produce while the SM streams one 64-column step of two G tiles
-// (about 0.6 us): the cluster is made large enough that a CTA's share of a tile stays below this.
-constexpr int PAIR_VALUES_PER_STEP = 2048;
 
 // Work decomposition of compress_pair_kernel (ranks above 64).
 //
@@ -233,8 +230,11 @@ inline void plan_compress_pair(TcSet& set, const std::vector<flora_mat>& G, int 
         max_tiles = std::max(max_tiles, tiles);
         total_work += tiles * ks;
     }
-    int S = 2;
-    while (S < 8 && N * 64 / S > PAIR_VALUES_PER_STEP) S <<= 1;
+    // Clusters of eight wherever the matrices have the rows for them: a slice of A then serves 2048 rows, and a 1600-row
+    // matrix is one unit (at N = 128 clusters of four keep a CTA's share of a slice within what its generators make
+    // during a step, and fit 132 SMs instead of 120, but generate every slice of such a matrix twice: 824 against 714 us
+    // on config 5's set at r = 128, 32.8 against 28.9 us on one 4096 x 11008 matrix).
+    int S = 8;
     while (S > 2 && (int64_t)S * T > 2 * max_tiles) S >>= 1;          // not more CTAs than there are rows to share
     S = tune_knob("FLORA_K1_CLUSTER", S, 2, 8);
     if (S & (S - 1)) S = 2;
@@ -245,6 +245,13 @@ inline void plan_compress_pair(TcSet& set, const std::vector<flora_mat>& G, int 
     // (five when that leaves fewer than three stages for G).  The G tiles come from HBM and get the rest.
     int astages = 6;
     if ((ring_budget - astages * a_stage) / g_stage < 3) astages = 5;
+    {
+        // ... and enough of them that sixteen generator warps and the epilogue warps can all hold a claim (see below):
+        // narrow slices (N = 128 in a cluster of eight: four work items per step) need up to eight stages of 8 KB
+        const int parts = (N / S * 8 + 31) / 32;
+        const int wanted = (PAIR_MAX_GEN_WARPS + PAIR_EPI_WARPS + parts - 1) / parts + 2;
+        while (astages < std::min(8, wanted) && (ring_budget - (astages + 1) * a_stage) / g_stage >= 3) ++astages;
+    }
     astages = tune_knob("FLORA_K1_ASTAGES", astages, 2, 8);
     int gstages = (int)std::min<size_t>(PAIR_RELAY_DEPTH - 1, (ring_budget - astages * a_stage) / g_stage);
     gstages = tune_knob("FLORA_K1_GSTAGES", std::max(1, gstages), 1, std::max(1, gstages));
